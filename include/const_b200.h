@@ -1,0 +1,192 @@
+/*
+ * const_b200 -- execution of fused sparse tensor-network contraction trees on one B200 GPU.
+ *
+ * The library runs the computation that the CoNST code generator emits (arXiv 2401.04836): a tree
+ * of binary contractions over CSF sparse tensors and dense factors, executed as one fused loop
+ * nest in which every intermediate keeps only the modes below the fused loops (Sec. 2.2, Fig. 4(b),
+ * Fig. 5).  The schedule -- contraction order, loop order of every contraction, CSF mode order of
+ * every sparse tensor (the ap / lp / dp values of Sec. 3.2) -- is an input; finding it is not part
+ * of this library.
+ *
+ * Conventions for every entry point
+ *   - C ABI, no exceptions, nothing is printed, nothing calls exit().
+ *   - "dev" pointers are CUDA device pointers on the current device; everything else is host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - The caller owns COO inputs, dense factors and outputs.  The library owns CSF arrays, work lists
+ *     and scratch (stream-ordered allocations on the given stream) until const_destroy.
+ *   - Dense operands and outputs are row-major in the index order written in the expression.
+ *   - Every function returns a const_status_t; on error no output handle is produced.
+ */
+#ifndef CONST_B200_H
+#define CONST_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CONST_OK = 0,
+    CONST_ERR_INVALID_ARG = 1,      /* null pointer, bad order, malformed expression ...               */
+    CONST_ERR_UNSUPPORTED = 2,      /* legal schedule that matches no kernel family, nnz >= 2^31 ...   */
+    CONST_ERR_ILLEGAL_SCHEDULE = 3, /* violates a constraint of Sec. 3.2                               */
+    CONST_ERR_DUPLICATE_COORD = 4,  /* the same coordinate tuple appears twice in a COO input          */
+    CONST_ERR_COORD_RANGE = 5,      /* a coordinate is negative or >= its extent                       */
+    CONST_ERR_WORKSPACE = 6,        /* a size exceeds a fixed internal capacity                        */
+    CONST_ERR_CUDA = 7,             /* a CUDA runtime call failed                                      */
+    CONST_ERR_TIMEOUT = 8           /* a bounded device-side wait gave up                              */
+} const_status_t;
+
+typedef enum { CONST_F32 = 0, CONST_F64 = 1 } const_dtype_t;
+
+typedef struct const_csf const_csf_t;     /* opaque: a sparse tensor in CSF form, on the device */
+typedef struct const_plan const_plan_t;   /* opaque: a checked schedule bound to a kernel family */
+
+typedef struct { char index; int64_t extent; } const_extent_t;   /* one per iteration index */
+
+/* One operand of const_execute: exactly one of `csf` / `dense_dev` is non-NULL. */
+typedef struct { const char *name; const const_csf_t *csf; const void *dense_dev; } const_operand_t;
+
+/*
+ * COO -> CSF (Sec. 2.1, "CSF representation").
+ *
+ * The tensor has `order` modes (2..4) with extents dims[0..order).  coords_dev[m] is a device array
+ * of nnz int32 coordinates of mode m; vals_dev holds nnz values of `dtype`.  The inputs are read,
+ * never modified, and may be released once the stream has passed this call.
+ * mode_order[l] is the mode stored at CSF level l (outermost first): the layout <d1,d2,d0> of the
+ * paper's example is mode_order = {1,2,0}.
+ *
+ * Result arrays (all int32, all levels compressed, nodes in lexicographic order):
+ *   crd[l][n]  coordinate of node n of level l;
+ *   pos[l][p]  first child (index into level l) of node p of level l-1, pos[l][n_{l-1}] = n_l;
+ *              pos[0] = {0, n_0};
+ *   vals[n]    value of leaf n (bit pattern untouched; explicit zeros are kept).
+ * The coordinate tuple is packed into one 64-bit key (sum of ceil(log2 extent) over modes must be
+ * <= 64), radix-sorted with its value, then each level is compressed with a flag/scan/scatter pass.
+ * Per-slice nonzero counts and the light / heavy / giant work lists used by const_execute are built
+ * here as well.
+ *
+ * Errors: CONST_ERR_COORD_RANGE, CONST_ERR_DUPLICATE_COORD (both detected on the device; the call
+ * synchronises the stream once to read sizes and status), CONST_ERR_UNSUPPORTED for nnz >= 2^31 - 1
+ * or a key wider than 64 bits, CONST_ERR_INVALID_ARG, CONST_ERR_CUDA.
+ */
+const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz,
+                               const int32_t *const *coords_dev, const void *vals_dev, const_dtype_t dtype,
+                               const int *mode_order, void *stream, const_csf_t **out);
+
+/* Borrowed device pointers of one level (valid until const_destroy).  *pos has n_{level-1}+1 entries
+ * (2 for level 0), *crd has *n entries.  Any output pointer may be NULL. */
+const_status_t const_csf_level(const const_csf_t *csf, int level, const int32_t **pos, const int32_t **crd,
+                               int64_t *n);
+/* Borrowed device pointer of the leaf values, in leaf order. */
+const_status_t const_csf_values(const const_csf_t *csf, const void **vals, int64_t *nnz);
+
+/*
+ * Load balancing over slices of the root level (work lists consumed by const_execute).
+ * A slice with at most light_max_nnz nonzeros is processed by one warp; up to heavy_max_nnz by one
+ * thread block; a larger ("giant") slice is split into blocks of about chunk_nnz nonzeros whose
+ * partial results are added atomically.  const_csf_build applies defaults; this call replaces them
+ * (used to force each bin in tests and to tune).  Values <= 0 keep the current setting.
+ */
+const_status_t const_csf_set_bins(const_csf_t *csf, int64_t light_max_nnz, int64_t heavy_max_nnz,
+                                  int64_t chunk_nnz, void *stream);
+/* Number of slices in each bin and of thread-block work items; any pointer may be NULL. */
+const_status_t const_csf_bin_counts(const const_csf_t *csf, int64_t *n_light, int64_t *n_heavy,
+                                    int64_t *n_giant, int64_t *n_items);
+
+/*
+ * Check a schedule and bind it to a kernel family (Sec. 3.1 input/output; Sec. 3.2 constraints;
+ * Sec. 4.2 the sequence of <assignment, loop permutation> pairs).
+ *
+ *   expression      the whole network, e.g. "Y[i,a,b] = X[i,j,k] * U[j,a] * V[k,b]".  Index names are
+ *                   single letters; tensor names are identifiers.
+ *   tree            n_contractions binary contractions in execution order (the ap order), e.g.
+ *                   "T[i,j,b] = X[i,j,k] * V[k,b]", "Y[i,a,b] = T[i,j,b] * U[j,a]".  The last one
+ *                   produces the result of `expression`.
+ *   sparse_names / mode_orders
+ *                   the n_sparse input tensors held in CSF and, for each, mode_orders[t][l] = mode at
+ *                   level l (dp).  Every other input is a dense row-major array.
+ *   loop_orders     one string per contraction: its indices, outermost loop first (lp).
+ *   extents         extent of every index that occurs.
+ *
+ * Checks (-> CONST_ERR_ILLEGAL_SCHEDULE): each contraction's operands are inputs or results of
+ * earlier contractions and every intermediate is consumed exactly once, later (Sec. 3.2.1); mode
+ * orders and loop orders are permutations (3.2.2, 3.2.3); each CSF operand's level order agrees with
+ * the loop order of the contraction that reads it, dense operands and dense-workspace intermediates
+ * being exempt (3.2.4); for each intermediate the loops shared as a common prefix by its producer,
+ * its consumer and every contraction between them are indices of the intermediate -- they are the
+ * modes fusion removes (3.2.5).  The tree must also compute `expression` (same inputs, same result
+ * indices, an index is summed in exactly one contraction).
+ *
+ * Kernel families (-> CONST_ERR_UNSUPPORTED otherwise):
+ *   chain   one CSF tensor of order 3 or 4 contracted leaf level first with one dense factor per
+ *           non-root level; the result is indexed by the root level followed by the rank indices in
+ *           level order (TTMc), or by one rank index shared by all factors (MTTKRP).  Ranks must be
+ *           8, 16 or 32 (order-4 TTMc: 8).  The loops above each contracted level must be fused, so
+ *           intermediates reduce to order 1 (order 2 for the middle one of order-4 TTMc).  CONST_F32.
+ *   network T[i,k,l] = U[i,j,k] * V[j,l]; Z[i,m] = T[i,k,l] * W[k,l,m] with V dense, U in CSF with
+ *           levels (i,k,j) and W in CSF with levels (m,l,k), loop orders i,k,j,l and i,m,l,k: both
+ *           contractions then gather along a fibre; fused over i only (T reduced to order 2).  CONST_F64.
+ */
+const_status_t const_plan_create(const char *expression, const char *const *tree, int n_contractions,
+                                 const char *const *sparse_names, const int *const *mode_orders, int n_sparse,
+                                 const char *const *loop_orders, const const_extent_t *extents, int n_indices,
+                                 const_dtype_t dtype, const_plan_t **out);
+
+/*
+ * The legality check of const_plan_create alone (Sec. 3.2), for any contraction tree, whether or not
+ * a kernel family exists for it.  On CONST_OK reduced_orders[c] (may be NULL) receives the order of
+ * the intermediate produced by contraction c after fusion (0 for the last contraction): its order
+ * minus the number of fused loops, the quantity the paper's parameter l bounds.  Host only.
+ */
+const_status_t const_schedule_check(const char *expression, const char *const *tree, int n_contractions,
+                                    const char *const *sparse_names, const int *const *mode_orders, int n_sparse,
+                                    const char *const *loop_orders, const const_extent_t *extents, int n_indices,
+                                    int *reduced_orders);
+
+/* Facts about a checked plan, for tests: reduced order of the intermediate produced by contraction
+ * c (0 for the last contraction), and the family ("ttmc3", "ttmc4", "mttkrp3", "network"). */
+const_status_t const_plan_reduced_order(const const_plan_t *plan, int contraction, int *order);
+const char *const_plan_family(const const_plan_t *plan);
+
+/*
+ * Run the fused contraction tree (Fig. 4(b) / Fig. 5 structure).  `operands` binds every input name
+ * of the expression to a CSF handle or a dense device array; CSF handles must have been built with
+ * the mode order and dtype the plan was created with.  out_dev is overwritten (it is zeroed first:
+ * "R[*] = 0" precedes the nest).  Asynchronous on `stream`; no host synchronisation.
+ * Partial results of split slices are combined with floating-point atomics, so results can differ
+ * in the last bits between runs.
+ */
+const_status_t const_execute(const_plan_t *plan, const const_operand_t *operands, int n_operands,
+                             void *out_dev, void *stream);
+
+/* Synchronise `stream` and return the device-side status word of the plan's last executions
+ * (CONST_OK, or the first error a kernel recorded, e.g. CONST_ERR_TIMEOUT). */
+const_status_t const_last_device_status(const_plan_t *plan, void *stream);
+
+/* Release a CSF handle or a plan (NULL is a no-op).  Device memory is freed in stream order on the
+ * stream the handle was built on. */
+void const_destroy(void *handle);
+
+const char *const_status_string(const_status_t status);
+
+/*
+ * Per-kernel timing (off by default).  While enabled, every kernel the library launches is
+ * bracketed by two CUDA events recorded on the launch stream.  const_profile_enable(1) also clears
+ * earlier records; const_profile_enable(0) stops recording and clears them.
+ * const_profile_read waits for the recorded events and returns, per kernel name in first-launch
+ * order, the number of launches and the summed duration in milliseconds.  `names` (host, may be
+ * NULL) receives the names separated by '\n'.  *n_kernels is the number of distinct names; at
+ * most max_kernels entries of `launches` / `total_ms` (host arrays, may be NULL) are written.
+ * Not thread-safe with respect to concurrent library calls on other threads beyond a mutex
+ * around the record list; meant for benchmarking, not for production paths.
+ */
+const_status_t const_profile_enable(int on);
+const_status_t const_profile_read(char *names, int64_t names_bytes, int64_t *launches, double *total_ms,
+                                  int max_kernels, int *n_kernels);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONST_B200_H */

@@ -1,0 +1,107 @@
+// Shared declarations of the CUDA library: handles, work items, small device helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <cstring>
+#include <string>
+
+#include "../../include/const_b200.h"
+#include "plan.h"
+
+namespace cb {
+
+constexpr uint32_t kCsfMagic = 0x31465343u;   // "CSF1"
+constexpr uint32_t kPlanMagic = 0x314e4c50u;  // "PLN1"
+constexpr int kMaxOrder = 4;
+
+// One thread-block work item of the fused kernels.
+//   kind 0: a group of light slices, one per warp: `slice` = first index into the light list, f0 = how many
+//   kind 1: a whole slice handled by one block: level-1 nodes [f0, f1); result stored directly
+//   kind 2: a chunk of a giant slice: level-1 nodes [f0, f1); result added atomically
+struct WorkItem {
+    int32_t slice;
+    int32_t f0;
+    int32_t f1;
+    int32_t kind;
+};
+
+constexpr int kItemLight = 0, kItemBlock = 1, kItemChunk = 2;
+constexpr int kWarpsPerBlock = 8;             // fused kernels run 256-thread blocks
+
+}  // namespace cb
+
+// The public opaque handles.
+struct const_csf {
+    uint32_t magic = cb::kCsfMagic;
+    int order = 0;
+    const_dtype_t dtype = CONST_F32;
+    int64_t dims[cb::kMaxOrder] = {0, 0, 0, 0};
+    int mode_order[cb::kMaxOrder] = {0, 0, 0, 0};
+    int64_t nnz = 0;
+    int64_t n[cb::kMaxOrder] = {0, 0, 0, 0};            // nodes per level
+    int32_t *pos[cb::kMaxOrder] = {nullptr, nullptr, nullptr, nullptr};
+    int32_t *crd[cb::kMaxOrder] = {nullptr, nullptr, nullptr, nullptr};
+    void *vals = nullptr;
+    // load balancing
+    int32_t *slice_ptr = nullptr;      // [n0 + 1] leaf offset of every root-level slice
+    int32_t *light_list = nullptr;     // [n_light] slice ids handled one per warp
+    cb::WorkItem *items = nullptr;     // [n_items]
+    int32_t *bin_scratch = nullptr;    // [2 * (n0 + 1) + 8] scan outputs
+    int64_t n_light = 0, n_heavy = 0, n_giant = 0, n_items = 0;
+    int64_t light_max = 0, heavy_max = 0, chunk = 0;
+    cudaStream_t stream = nullptr;
+    int device = 0;
+};
+
+struct const_plan {
+    uint32_t magic = cb::kPlanMagic;
+    cb::PlanDesc desc;
+    int32_t *status_dev = nullptr;     // device status word written by kernels
+    int device = -1;
+};
+
+namespace cb {
+
+#define CB_CUDA(call)                                         \
+    do {                                                      \
+        cudaError_t _e = (call);                              \
+        if (_e != cudaSuccess) return CONST_ERR_CUDA;         \
+    } while (0)
+
+// profile.cu: brackets a kernel launch with two events when profiling is on (no-op otherwise)
+class ProfScope {
+public:
+    ProfScope(const char *name, cudaStream_t stream);
+    ~ProfScope();
+    ProfScope(const ProfScope &) = delete;
+    ProfScope &operator=(const ProfScope &) = delete;
+private:
+    cudaStream_t stream_;
+    long idx_;
+};
+#define CB_LAUNCH(name, stream, ...)             \
+    do {                                         \
+        cb::ProfScope _prof(name, stream);       \
+        __VA_ARGS__;                             \
+    } while (0)
+
+// csf_build.cu
+const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
+                              const void *vals_dev, const_dtype_t dtype, const int *mode_order,
+                              cudaStream_t stream, const_csf **out);
+const_status_t csf_rebin(const_csf *csf, cudaStream_t stream);
+void csf_free(const_csf *csf);
+
+// chain_kernels.cu
+const_status_t run_ttmc3(const const_csf *X, const float *U, const float *V, int R2, int R3, float *Y,
+                         int64_t n_rows, int32_t *status, cudaStream_t stream);
+const_status_t run_mttkrp3(const const_csf *X, const float *B, const float *C, int R, float *A,
+                           int64_t n_rows, int32_t *status, cudaStream_t stream);
+const_status_t run_ttmc4(const const_csf *X, const float *U, const float *V, const float *W, int R, float *Y,
+                         int64_t n_rows, int32_t *status, cudaStream_t stream);
+// network_kernels.cu
+const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z,
+                           int64_t n_i, int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m,
+                           int32_t *status, cudaStream_t stream);
+
+}  // namespace cb

@@ -1,0 +1,724 @@
+// GPU CSF builder (Sec. 2.1, CSF representation): pack -> LSD radix sort -> per-level compression,
+// followed by the per-slice load-balancing lists used by the fused contraction kernels.
+//
+// Layout decisions
+//   * The permuted coordinate tuple is packed into one 64-bit key, root level in the top bits, so a
+//     single key sort orders the nonzeros lexicographically by the chosen mode order.
+//   * The value travels with its key as the sort payload, so no gather pass is needed afterwards and
+//     the sorted payload buffer *is* the leaf value array.
+//   * The sort is a least-significant-digit radix sort with 8-bit digits.  Each pass is one kernel:
+//     tiles are ranked in shared memory, the tile's digit counts are chained to earlier tiles with a
+//     decoupled look-back (every spin is bounded and reports CONST_ERR_TIMEOUT), and keys are
+//     reordered in shared memory so that global stores run over consecutive addresses.
+//   * Compression is flag / scan / scatter: element e opens a node at level l when its length-(l+1)
+//     prefix differs from that of e-1.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace cb {
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// pack
+// ------------------------------------------------------------------------------------------------
+struct PackArgs {
+    const int32_t *c[kMaxOrder];   // coordinates of the mode stored at level l
+    int64_t dim[kMaxOrder];
+    int shift[kMaxOrder];
+    int order;
+};
+
+enum DevErr : int32_t { kErrNone = 0 };
+
+__device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicCAS(status, 0, code); }
+
+__global__ void pack_keys(PackArgs a, int64_t nnz, uint64_t *__restrict__ keys, int32_t *status) {
+    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= nnz) return;
+    uint64_t key = 0;
+    bool bad = false;
+    for (int l = 0; l < a.order; ++l) {
+        int64_t c = a.c[l][e];
+        if (c < 0 || c >= a.dim[l]) { bad = true; c = 0; }
+        key |= (uint64_t)c << a.shift[l];
+    }
+    if (bad) report(status, CONST_ERR_COORD_RANGE);
+    keys[e] = key;
+}
+
+// ------------------------------------------------------------------------------------------------
+// radix sort
+// ------------------------------------------------------------------------------------------------
+constexpr int kRsBins = 256;
+constexpr int kRsThreads = 256;
+constexpr int kRsItems = 16;
+constexpr int kRsTile = kRsThreads * kRsItems;     // 4096 keys per tile
+constexpr int kRsWarps = kRsThreads / 32;
+constexpr int kMaxPasses = 8;
+constexpr uint64_t kFlagAgg = 1ull << 62;          // tile published its own digit counts
+constexpr uint64_t kFlagInc = 2ull << 62;          // tile published counts summed over all earlier tiles too
+constexpr uint64_t kValMask = (1ull << 62) - 1;
+constexpr int kSpinLimit = 1 << 21;
+
+// Digit histograms of every pass in one read of the keys.
+__global__ void __launch_bounds__(256) rs_histogram(const uint64_t *__restrict__ keys, int64_t n, int passes,
+                                                    uint32_t *__restrict__ hist) {
+    __shared__ uint32_t sh[kMaxPasses * kRsBins];
+    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x) sh[x] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x; base < n; base += stride) {   // base is block-uniform
+        int64_t e = base + threadIdx.x;
+        bool valid = e < n;
+        unsigned active = __ballot_sync(0xffffffffu, valid);
+        if (valid) {
+            uint64_t key = keys[e];
+            for (int p = 0; p < passes; ++p) {
+                unsigned d = (unsigned)(key >> (8 * p)) & 255u;
+                unsigned peers = __match_any_sync(active, d);
+                if (lane == __ffs(peers) - 1) atomicAdd(&sh[p * kRsBins + d], __popc(peers));
+            }
+        }
+    }
+    __syncthreads();
+    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x)
+        if (sh[x]) atomicAdd(&hist[x], sh[x]);
+}
+
+// Exclusive scan of each pass's 256-bin histogram: one block per pass.
+__global__ void __launch_bounds__(256) rs_scan_hist(uint32_t *hist) {
+    __shared__ uint32_t sh[kRsBins];
+    uint32_t *h = hist + blockIdx.x * kRsBins;
+    sh[threadIdx.x] = h[threadIdx.x];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t run = 0;
+        for (int d = 0; d < kRsBins; ++d) { uint32_t c = sh[d]; sh[d] = run; run += c; }
+    }
+    __syncthreads();
+    h[threadIdx.x] = sh[threadIdx.x];
+}
+
+template <typename V>
+__global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__restrict__ kin, uint64_t *__restrict__ kout,
+                                                         const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
+                                                         int shift, const uint32_t *__restrict__ digit_base,
+                                                         unsigned long long *status, uint32_t *counter,
+                                                         int32_t *err) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t *keybuf = reinterpret_cast<uint64_t *>(smem_raw);
+    V *valbuf = reinterpret_cast<V *>(smem_raw + kRsTile * sizeof(uint64_t));
+    __shared__ uint32_t warp_hist[kRsWarps][kRsBins];
+    __shared__ uint32_t digit_excl[kRsBins];
+    __shared__ long long s_gbase[kRsBins];
+    __shared__ uint32_t warp_tot[kRsWarps];
+    __shared__ uint32_t s_tile;
+    __shared__ int s_abort;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { s_tile = atomicAdd(counter, 1u); s_abort = 0; }
+    for (int x = threadIdx.x; x < kRsWarps * kRsBins; x += kRsThreads) (&warp_hist[0][0])[x] = 0;
+    __syncthreads();
+    const int64_t tile = s_tile;
+    const int64_t tile_base = tile * kRsTile;
+    if (tile_base >= n) return;                       // never happens: the grid has exactly ceil(n / tile) blocks
+
+    uint64_t key[kRsItems];
+    V val[kRsItems];
+#pragma unroll
+    for (int i = 0; i < kRsItems; ++i) {
+        int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
+        bool in = idx < n;
+        key[i] = in ? kin[idx] : ~0ull;               // padding sorts after every real key of the tile
+        val[i] = in ? vin[idx] : V(0);
+    }
+
+    // rank inside the warp: keys with equal digits keep their order (item, lane)
+    int rank[kRsItems];
+#pragma unroll
+    for (int i = 0; i < kRsItems; ++i) {
+        unsigned d = (unsigned)(key[i] >> shift) & 255u;
+        unsigned peers = __match_any_sync(0xffffffffu, d);
+        int leader = __ffs(peers) - 1;
+        uint32_t old = 0;
+        if (lane == leader) {
+            old = warp_hist[warp][d];
+            warp_hist[warp][d] = old + __popc(peers);
+        }
+        old = __shfl_sync(0xffffffffu, old, leader);
+        rank[i] = (int)old + __popc(peers & ((1u << lane) - 1u));
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // thread d owns digit d: offsets of each warp's run, tile total, digit scan inside the tile
+    const int d = threadIdx.x;
+    uint32_t count = 0;
+#pragma unroll
+    for (int w = 0; w < kRsWarps; ++w) {
+        uint32_t c = warp_hist[w][d];
+        warp_hist[w][d] = count;
+        count += c;
+    }
+    uint32_t incl = count;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        uint32_t v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    uint32_t wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += warp_tot[w];
+    const uint32_t excl_in_tile = wbase + incl - count;
+
+    // chained scan over tiles (decoupled look-back); every wait is bounded
+    volatile unsigned long long *st = status;
+    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | (unsigned long long)count;
+    unsigned long long before = 0;
+    if (tile > 0) {
+        bool ok = true;
+        int64_t t = tile - 1;
+        for (;;) {
+            unsigned long long s = 0;
+            int spins = 0;
+            for (;;) {
+                s = st[t * kRsBins + d];
+                if (s >> 62) break;
+                if (++spins > kSpinLimit) { ok = false; break; }
+                if (spins > 64) __nanosleep(100);
+            }
+            if (!ok) break;
+            before += s & kValMask;
+            if ((s >> 62) == 2ull || t == 0) break;
+            --t;
+        }
+        if (ok) {
+            st[tile * kRsBins + d] = kFlagInc | (before + count);
+        } else {
+            report(err, CONST_ERR_TIMEOUT);
+            s_abort = 1;
+        }
+    }
+    digit_excl[d] = excl_in_tile;
+    s_gbase[d] = (long long)digit_base[d] + (long long)before - (long long)excl_in_tile;
+    __syncthreads();
+    if (s_abort) return;
+
+    // reorder in shared memory, then store runs of consecutive addresses
+#pragma unroll
+    for (int i = 0; i < kRsItems; ++i) {
+        unsigned dg = (unsigned)(key[i] >> shift) & 255u;
+        int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
+        keybuf[p] = key[i];
+        valbuf[p] = val[i];
+    }
+    __syncthreads();
+    const int64_t left = n - tile_base;
+    const int nvalid = left < kRsTile ? (int)left : kRsTile;
+#pragma unroll
+    for (int m = 0; m < kRsItems; ++m) {
+        int p = threadIdx.x + m * kRsThreads;
+        if (p < nvalid) {
+            uint64_t k = keybuf[p];
+            unsigned dg = (unsigned)(k >> shift) & 255u;
+            long long o = s_gbase[dg] + p;
+            kout[o] = k;
+            vout[o] = valbuf[p];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// compression: flags -> counts -> scan -> scatter
+// ------------------------------------------------------------------------------------------------
+constexpr int kCpThreads = 256;
+constexpr int kCpIters = 8;                                   // 32-element steps per warp
+constexpr int kCpTile = kCpThreads * kCpIters;                // 2048 elements per block
+constexpr int kCpLevels = kMaxOrder - 1;                      // levels that need a scan (all but the leaf level)
+
+struct LevelShifts { int shift[kMaxOrder]; int order; };
+
+// ballots of "opens a new node at level l" for the 32 elements starting at `base`
+__device__ __forceinline__ void node_flags(const uint64_t *__restrict__ keys, int64_t n, int64_t base, int lane,
+                                           const LevelShifts &ls, uint64_t &key, unsigned ballots[kCpLevels],
+                                           bool &dup) {
+    int64_t e = base + lane;
+    bool in = e < n;
+    key = in ? keys[e] : 0ull;
+    uint64_t prev = __shfl_up_sync(0xffffffffu, key, 1);
+    if (lane == 0 && in && e > 0) prev = keys[e - 1];
+    bool first = (e == 0);
+    dup = in && !first && key == prev;
+#pragma unroll
+    for (int l = 0; l < kCpLevels; ++l) {
+        bool f = false;
+        if (l < ls.order - 1) f = in && (first || (key >> ls.shift[l]) != (prev >> ls.shift[l]));
+        ballots[l] = __ballot_sync(0xffffffffu, f);
+    }
+}
+
+__global__ void __launch_bounds__(kCpThreads) csf_count(const uint64_t *__restrict__ keys, int64_t n, LevelShifts ls,
+                                                       uint32_t *__restrict__ block_counts, int32_t *status) {
+    __shared__ uint32_t sh[kCpLevels];
+    if (threadIdx.x < kCpLevels) sh[threadIdx.x] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t cnt[kCpLevels] = {0, 0, 0};
+    bool any_dup = false;
+    for (int it = 0; it < kCpIters; ++it) {
+        int64_t base = (int64_t)blockIdx.x * kCpTile + (warp * kCpIters + it) * 32;
+        uint64_t key; unsigned b[kCpLevels]; bool dup;
+        node_flags(keys, n, base, lane, ls, key, b, dup);
+        any_dup |= dup;
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) cnt[l] += __popc(b[l]);
+    }
+    if (any_dup) report(status, CONST_ERR_DUPLICATE_COORD);
+    if (lane == 0)
+        for (int l = 0; l < kCpLevels; ++l) atomicAdd(&sh[l], cnt[l]);
+    __syncthreads();
+    if (threadIdx.x < kCpLevels) block_counts[(int64_t)blockIdx.x * kCpLevels + threadIdx.x] = sh[threadIdx.x];
+}
+
+// In-place exclusive scan of per-block counts (one block); totals[l] receives the level sizes.
+__global__ void __launch_bounds__(1024) csf_scan_blocks(uint32_t *block_counts, int64_t nblocks, uint32_t *totals) {
+    __shared__ uint32_t wsum[32][kCpLevels];
+    __shared__ uint32_t carry[kCpLevels];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < kCpLevels) carry[threadIdx.x] = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < nblocks; base += 1024) {
+        int64_t b = base + threadIdx.x;
+        uint32_t v[kCpLevels], inc[kCpLevels];
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) {
+            v[l] = b < nblocks ? block_counts[b * kCpLevels + l] : 0;
+            inc[l] = v[l];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                uint32_t t = __shfl_up_sync(0xffffffffu, inc[l], off);
+                if (lane >= off) inc[l] += t;
+            }
+            if (lane == 31) wsum[warp][l] = inc[l];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) {
+            uint32_t wb = 0;
+            for (int w = 0; w < warp; ++w) wb += wsum[w][l];
+            if (b < nblocks) block_counts[b * kCpLevels + l] = carry[l] + wb + inc[l] - v[l];
+        }
+        __syncthreads();
+        if (threadIdx.x == 1023)
+            for (int l = 0; l < kCpLevels; ++l) {
+                uint32_t wb = 0;
+                for (int w = 0; w < 31; ++w) wb += wsum[w][l];
+                carry[l] += wb + inc[l];
+            }
+        __syncthreads();
+    }
+    if (threadIdx.x < kCpLevels) totals[threadIdx.x] = carry[threadIdx.x];
+}
+
+struct CsfArrays {
+    int32_t *pos[kMaxOrder];
+    int32_t *crd[kMaxOrder];
+    int bits[kMaxOrder];
+};
+
+__global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__restrict__ keys, int64_t n, LevelShifts ls,
+                                                         const uint32_t *__restrict__ block_base, CsfArrays out) {
+    __shared__ uint32_t wcnt[kCpThreads / 32][kCpLevels];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint64_t key[kCpIters];
+    unsigned bal[kCpIters][kCpLevels];
+    uint32_t cnt[kCpLevels] = {0, 0, 0};
+#pragma unroll
+    for (int it = 0; it < kCpIters; ++it) {
+        int64_t base = (int64_t)blockIdx.x * kCpTile + (warp * kCpIters + it) * 32;
+        bool dup;
+        node_flags(keys, n, base, lane, ls, key[it], bal[it], dup);
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) cnt[l] += __popc(bal[it][l]);
+    }
+    if (lane == 0)
+        for (int l = 0; l < kCpLevels; ++l) wcnt[warp][l] = cnt[l];
+    __syncthreads();
+    uint32_t run[kCpLevels];
+#pragma unroll
+    for (int l = 0; l < kCpLevels; ++l) {
+        run[l] = block_base[(int64_t)blockIdx.x * kCpLevels + l];
+        for (int w = 0; w < warp; ++w) run[l] += wcnt[w][l];
+    }
+    const int leaf = ls.order - 1;
+    const unsigned below = (1u << lane) - 1u;
+#pragma unroll
+    for (int it = 0; it < kCpIters; ++it) {
+        int64_t e = (int64_t)blockIdx.x * kCpTile + (warp * kCpIters + it) * 32 + lane;
+        if (e < n) {
+            uint32_t id[kMaxOrder];
+#pragma unroll
+            for (int l = 0; l < kCpLevels; ++l) id[l] = run[l] + __popc(bal[it][l] & below);
+            id[leaf] = (uint32_t)e;
+            out.crd[leaf][e] = (int32_t)((key[it] >> ls.shift[leaf]) & ((1ull << out.bits[leaf]) - 1ull));
+#pragma unroll
+            for (int l = 0; l < kCpLevels; ++l) {
+                if (l < leaf && ((bal[it][l] >> lane) & 1u)) {
+                    out.crd[l][id[l]] = (int32_t)((key[it] >> ls.shift[l]) & ((1ull << out.bits[l]) - 1ull));
+                    out.pos[l + 1][id[l]] = (int32_t)id[l + 1];
+                }
+            }
+        }
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) run[l] += __popc(bal[it][l]);
+    }
+}
+
+struct LevelSizes { int64_t n[kMaxOrder]; int order; };
+
+__global__ void csf_finish(CsfArrays out, LevelSizes sz) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        out.pos[0][0] = 0;
+        out.pos[0][1] = (int32_t)sz.n[0];
+        for (int l = 1; l < sz.order; ++l) out.pos[l][sz.n[l - 1]] = (int32_t)sz.n[l];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// load balancing (per-slice nonzero counts -> light / heavy / giant work lists)
+// ------------------------------------------------------------------------------------------------
+struct ChainPtrs { const int32_t *pos[kMaxOrder]; int order; };
+
+// leaf offset of level-1 node f (or of the end when f = n1)
+__device__ __forceinline__ int32_t leaf_of_fiber(const ChainPtrs &c, int32_t f) {
+    int32_t x = f;
+    for (int l = 2; l < c.order; ++l) x = c.pos[l][x];
+    return x;
+}
+
+__global__ void bin_slice_ptr(ChainPtrs c, int64_t n0, int32_t *__restrict__ slice_ptr) {
+    int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s > n0) return;
+    slice_ptr[s] = leaf_of_fiber(c, c.pos[1][s]);
+}
+
+// Single-block scan over slices: per-slice work-item offset and light-list index; totals in out[0..4).
+__global__ void __launch_bounds__(1024) bin_scan(const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t light_max,
+                                                 int64_t heavy_max, int64_t chunk, int32_t *__restrict__ item_off,
+                                                 int32_t *__restrict__ light_idx, int32_t *__restrict__ totals) {
+    __shared__ uint32_t wsum[32][2];
+    __shared__ uint32_t carry[4];      // items, light, heavy, giant
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < 4) carry[threadIdx.x] = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < n0; base += 1024) {
+        int64_t s = base + threadIdx.x;
+        uint32_t v[2] = {0, 0};
+        uint32_t is_heavy = 0, is_giant = 0;
+        if (s < n0) {
+            int64_t z = (int64_t)slice_ptr[s + 1] - slice_ptr[s];
+            if (z <= light_max) v[1] = 1;
+            else if (z <= heavy_max) { v[0] = 1; is_heavy = 1; }
+            else { v[0] = (uint32_t)((z + chunk - 1) / chunk); is_giant = 1; }
+        }
+        uint32_t inc[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            inc[q] = v[q];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                uint32_t t = __shfl_up_sync(0xffffffffu, inc[q], off);
+                if (lane >= off) inc[q] += t;
+            }
+            if (lane == 31) wsum[warp][q] = inc[q];
+        }
+        unsigned hb = __ballot_sync(0xffffffffu, is_heavy), gb = __ballot_sync(0xffffffffu, is_giant);
+        __syncthreads();
+        uint32_t wb[2] = {0, 0};
+        for (int w = 0; w < warp; ++w) { wb[0] += wsum[w][0]; wb[1] += wsum[w][1]; }
+        if (s < n0) {
+            item_off[s] = (int32_t)(carry[0] + wb[0] + inc[0] - v[0]);
+            light_idx[s] = (int32_t)(carry[1] + wb[1] + inc[1] - v[1]);
+        }
+        __syncthreads();
+        if (lane == 0) { atomicAdd(&carry[2], __popc(hb)); atomicAdd(&carry[3], __popc(gb)); }
+        if (threadIdx.x == 1023) { carry[0] += wb[0] + inc[0]; carry[1] += wb[1] + inc[1]; }
+        __syncthreads();
+    }
+    if (threadIdx.x < 4) totals[threadIdx.x] = (int32_t)carry[threadIdx.x];
+}
+
+__global__ void bin_fill(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t light_max,
+                         int64_t heavy_max, int64_t chunk, const int32_t *__restrict__ item_off,
+                         const int32_t *__restrict__ light_idx, WorkItem *__restrict__ items,
+                         int32_t *__restrict__ light_list) {
+    int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n0) return;
+    const int32_t p0 = slice_ptr[s], p1 = slice_ptr[s + 1];
+    const int64_t z = (int64_t)p1 - p0;
+    const int32_t f0 = c.pos[1][s], f1 = c.pos[1][s + 1];
+    if (z <= light_max) {
+        light_list[light_idx[s]] = (int32_t)s;
+    } else if (z <= heavy_max) {
+        items[item_off[s]] = WorkItem{(int32_t)s, f0, f1, kItemBlock};
+    } else {
+        const int64_t parts = (z + chunk - 1) / chunk;
+        int32_t begin = f0;
+        for (int64_t q = 0; q < parts; ++q) {
+            int32_t end = f1;
+            if (q + 1 < parts) {
+                // first level-1 node whose leaf offset reaches the target
+                const int64_t target = p0 + (z * (q + 1)) / parts;
+                int32_t lo = begin, hi = f1;
+                while (lo < hi) {
+                    int32_t mid = lo + (hi - lo) / 2;
+                    if ((int64_t)leaf_of_fiber(c, mid) < target) lo = mid + 1; else hi = mid;
+                }
+                end = lo;
+            }
+            items[item_off[s] + q] = WorkItem{(int32_t)s, begin, end, kItemChunk};
+            begin = end;
+        }
+    }
+}
+
+__global__ void bin_light_items(WorkItem *__restrict__ items, int64_t first_item, int64_t n_light) {
+    int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int64_t groups = (n_light + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (g >= groups) return;
+    int64_t left = n_light - g * kWarpsPerBlock;
+    items[first_item + g] = WorkItem{(int32_t)(g * kWarpsPerBlock),
+                                     (int32_t)(left < kWarpsPerBlock ? left : kWarpsPerBlock), 0, kItemLight};
+}
+
+int bits_for(int64_t extent) {
+    int b = 1;
+    while (b < 63 && (1ll << b) < extent) ++b;
+    return b;
+}
+
+struct Scratch {            // stream-ordered temporaries of one build
+    cudaStream_t stream;
+    void *ptrs[16];
+    int n = 0;
+    explicit Scratch(cudaStream_t s) : stream(s) {}
+    cudaError_t alloc(void **p, size_t bytes) {
+        cudaError_t e = cudaMallocAsync(p, bytes ? bytes : 16, stream);
+        if (e == cudaSuccess) ptrs[n++] = *p;
+        return e;
+    }
+    void forget(void *p) {
+        for (int i = 0; i < n; ++i) if (ptrs[i] == p) ptrs[i] = nullptr;
+    }
+    ~Scratch() {
+        for (int i = 0; i < n; ++i) if (ptrs[i]) cudaFreeAsync(ptrs[i], stream);
+    }
+};
+
+template <typename V>
+const_status_t sort_pairs(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
+                          Scratch &tmp, int32_t *status, cudaStream_t stream) {
+    if (n == 0 || passes == 0) return CONST_OK;
+    uint32_t *hist = nullptr, *counters = nullptr;
+    unsigned long long *tile_status = nullptr;
+    const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
+    CB_CUDA(tmp.alloc((void **)&hist, sizeof(uint32_t) * kMaxPasses * kRsBins));
+    CB_CUDA(tmp.alloc((void **)&counters, sizeof(uint32_t) * kMaxPasses));
+    CB_CUDA(tmp.alloc((void **)&tile_status, sizeof(unsigned long long) * ntiles * kRsBins));
+    CB_CUDA(cudaMemsetAsync(hist, 0, sizeof(uint32_t) * kMaxPasses * kRsBins, stream));
+    CB_CUDA(cudaMemsetAsync(counters, 0, sizeof(uint32_t) * kMaxPasses, stream));
+    int hist_blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    CB_LAUNCH("rs_histogram", stream, rs_histogram<<<hist_blocks, 256, 0, stream>>>(keys, n, passes, hist));
+    CB_LAUNCH("rs_scan_hist", stream, rs_scan_hist<<<passes, 256, 0, stream>>>(hist));
+    const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
+    CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    for (int p = 0; p < passes; ++p) {
+        CB_CUDA(cudaMemsetAsync(tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
+        CB_LAUNCH("rs_onesweep", stream, rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(keys, keys_alt, vals, vals_alt, n, 8 * p,
+                                                                     hist + p * kRsBins, tile_status, counters + p,
+                                                                     status));
+        std::swap(keys, keys_alt);
+        std::swap(vals, vals_alt);
+    }
+    CB_CUDA(cudaGetLastError());
+    return CONST_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// host driver
+// ------------------------------------------------------------------------------------------------
+void csf_free(const_csf *csf) {
+    if (!csf) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(csf->device);
+    auto drop = [&](void *p) { if (p) cudaFreeAsync(p, csf->stream); };
+    for (int l = 0; l < kMaxOrder; ++l) { drop(csf->pos[l]); drop(csf->crd[l]); }
+    drop(csf->vals);
+    drop(csf->slice_ptr);
+    drop(csf->light_list);
+    drop(csf->items);
+    drop(csf->bin_scratch);
+    csf->magic = 0;
+    delete csf;
+    cudaSetDevice(prev);
+}
+
+const_status_t csf_rebin(const_csf *csf, cudaStream_t stream) {
+    const int64_t n0 = csf->n[0];
+    if (csf->light_list) { cudaFreeAsync(csf->light_list, stream); csf->light_list = nullptr; }
+    if (csf->items) { cudaFreeAsync(csf->items, stream); csf->items = nullptr; }
+    csf->n_light = csf->n_heavy = csf->n_giant = csf->n_items = 0;
+    if (n0 == 0) return CONST_OK;
+    ChainPtrs c;
+    c.order = csf->order;
+    for (int l = 0; l < kMaxOrder; ++l) c.pos[l] = csf->pos[l];
+    int32_t *item_off = csf->bin_scratch, *light_idx = csf->bin_scratch + (n0 + 1), *totals = csf->bin_scratch + 2 * (n0 + 1);
+    CB_LAUNCH("bin_scan", stream, bin_scan<<<1, 1024, 0, stream>>>(csf->slice_ptr, n0, csf->light_max, csf->heavy_max, csf->chunk, item_off,
+                                     light_idx, totals));
+    int32_t h[4];
+    CB_CUDA(cudaMemcpyAsync(h, totals, sizeof(h), cudaMemcpyDeviceToHost, stream));
+    CB_CUDA(cudaStreamSynchronize(stream));
+    const int64_t hg_items = h[0];
+    csf->n_light = h[1];
+    csf->n_heavy = h[2];
+    csf->n_giant = h[3];
+    const int64_t light_groups = (csf->n_light + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    csf->n_items = hg_items + light_groups;
+    CB_CUDA(cudaMallocAsync((void **)&csf->items, sizeof(WorkItem) * std::max<int64_t>(csf->n_items, 1), stream));
+    CB_CUDA(cudaMallocAsync((void **)&csf->light_list, sizeof(int32_t) * std::max<int64_t>(csf->n_light, 1), stream));
+    CB_LAUNCH("bin_fill", stream, bin_fill<<<(unsigned)((n0 + 255) / 256), 256, 0, stream>>>(c, csf->slice_ptr, n0, csf->light_max, csf->heavy_max,
+                                                              csf->chunk, item_off, light_idx, csf->items,
+                                                              csf->light_list));
+    if (light_groups > 0)
+        CB_LAUNCH("bin_light_items", stream, bin_light_items<<<(unsigned)((light_groups + 255) / 256), 256, 0, stream>>>(csf->items, hg_items, csf->n_light));
+    CB_CUDA(cudaGetLastError());
+    return CONST_OK;
+}
+
+const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
+                              const void *vals_dev, const_dtype_t dtype, const int *mode_order,
+                              cudaStream_t stream, const_csf **out) {
+    // level layout of the packed key
+    int bits[kMaxOrder] = {0, 0, 0, 0}, shift[kMaxOrder] = {0, 0, 0, 0};
+    int total_bits = 0;
+    for (int l = 0; l < order; ++l) { bits[l] = bits_for(dims[mode_order[l]]); total_bits += bits[l]; }
+    if (total_bits > 64) return CONST_ERR_UNSUPPORTED;
+    int acc = 0;
+    for (int l = order - 1; l >= 0; --l) { shift[l] = acc; acc += bits[l]; }
+    const int passes = (total_bits + 7) / 8;
+
+    const_csf *csf = new (std::nothrow) const_csf();
+    if (!csf) return CONST_ERR_INVALID_ARG;
+    csf->order = order;
+    csf->dtype = dtype;
+    csf->nnz = nnz;
+    csf->stream = stream;
+    cudaGetDevice(&csf->device);
+    for (int l = 0; l < order; ++l) { csf->dims[l] = dims[l]; csf->mode_order[l] = mode_order[l]; }
+    csf->light_max = 1024;
+    csf->heavy_max = 49152;
+    csf->chunk = 24576;
+
+    const size_t vsize = dtype == CONST_F32 ? 4 : 8;
+    const_status_t rc = CONST_OK;
+    {
+        Scratch tmp(stream);
+        uint64_t *keys = nullptr, *keys_alt = nullptr;
+        void *vals = nullptr, *vals_alt = nullptr;
+        int32_t *status = nullptr;
+        uint32_t *block_counts = nullptr, *totals = nullptr;
+        const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
+        auto body = [&]() -> const_status_t {
+            CB_CUDA(tmp.alloc((void **)&keys, sizeof(uint64_t) * nnz));
+            CB_CUDA(tmp.alloc((void **)&keys_alt, sizeof(uint64_t) * nnz));
+            CB_CUDA(tmp.alloc(&vals, vsize * nnz));
+            CB_CUDA(tmp.alloc(&vals_alt, vsize * nnz));
+            CB_CUDA(tmp.alloc((void **)&status, sizeof(int32_t)));
+            CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * kCpLevels * std::max<int64_t>(cp_blocks, 1)));
+            CB_CUDA(tmp.alloc((void **)&totals, sizeof(uint32_t) * 4));
+            CB_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+            CB_CUDA(cudaMemsetAsync(totals, 0, sizeof(uint32_t) * 4, stream));
+            LevelShifts ls;
+            ls.order = order;
+            for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = shift[l];
+            if (nnz > 0) {
+                PackArgs pa;
+                pa.order = order;
+                for (int l = 0; l < kMaxOrder; ++l) {
+                    pa.c[l] = l < order ? coords_dev[mode_order[l]] : nullptr;
+                    pa.dim[l] = l < order ? dims[mode_order[l]] : 0;
+                    pa.shift[l] = shift[l];
+                }
+                CB_LAUNCH("pack_keys", stream, pack_keys<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(pa, nnz, keys, status));
+                CB_CUDA(cudaMemcpyAsync(vals, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
+                const_status_t s;
+                if (dtype == CONST_F32) {
+                    uint32_t *v = (uint32_t *)vals, *va = (uint32_t *)vals_alt;
+                    s = sort_pairs<uint32_t>(keys, keys_alt, v, va, nnz, passes, tmp, status, stream);
+                    vals = v; vals_alt = va;
+                } else {
+                    unsigned long long *v = (unsigned long long *)vals, *va = (unsigned long long *)vals_alt;
+                    s = sort_pairs<unsigned long long>(keys, keys_alt, v, va, nnz, passes, tmp, status, stream);
+                    vals = v; vals_alt = va;
+                }
+                if (s != CONST_OK) return s;
+                CB_LAUNCH("csf_count", stream, csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status));
+                CB_LAUNCH("csf_scan_blocks", stream, csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals));
+            }
+            uint32_t h_totals[4] = {0, 0, 0, 0};
+            int32_t h_status = 0;
+            CB_CUDA(cudaMemcpyAsync(h_totals, totals, sizeof(h_totals), cudaMemcpyDeviceToHost, stream));
+            CB_CUDA(cudaMemcpyAsync(&h_status, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+            CB_CUDA(cudaStreamSynchronize(stream));
+            if (h_status != 0) return (const_status_t)h_status;
+            for (int l = 0; l < order - 1; ++l) csf->n[l] = h_totals[l];
+            csf->n[order - 1] = nnz;
+
+            CsfArrays arr;
+            for (int l = 0; l < kMaxOrder; ++l) { arr.pos[l] = arr.crd[l] = nullptr; arr.bits[l] = bits[l]; }
+            for (int l = 0; l < order; ++l) {
+                const int64_t parents = l == 0 ? 1 : csf->n[l - 1];
+                CB_CUDA(cudaMallocAsync((void **)&csf->pos[l], sizeof(int32_t) * (parents + 1), stream));
+                CB_CUDA(cudaMallocAsync((void **)&csf->crd[l], sizeof(int32_t) * std::max<int64_t>(csf->n[l], 1), stream));
+                arr.pos[l] = csf->pos[l];
+                arr.crd[l] = csf->crd[l];
+            }
+            if (nnz > 0)
+                CB_LAUNCH("csf_scatter", stream, csf_scatter<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, arr));
+            LevelSizes sz;
+            sz.order = order;
+            for (int l = 0; l < kMaxOrder; ++l) sz.n[l] = csf->n[l];
+            CB_LAUNCH("csf_finish", stream, csf_finish<<<1, 32, 0, stream>>>(arr, sz));
+            csf->vals = vals;                 // the sorted payload buffer becomes the leaf value array
+            tmp.forget(vals);
+
+            // per-slice leaf offsets and the default work lists
+            const int64_t n0 = csf->n[0];
+            CB_CUDA(cudaMallocAsync((void **)&csf->slice_ptr, sizeof(int32_t) * (n0 + 1), stream));
+            CB_CUDA(cudaMallocAsync((void **)&csf->bin_scratch, sizeof(int32_t) * (2 * (n0 + 1) + 8), stream));
+            ChainPtrs c;
+            c.order = order;
+            for (int l = 0; l < kMaxOrder; ++l) c.pos[l] = csf->pos[l];
+            CB_LAUNCH("bin_slice_ptr", stream, bin_slice_ptr<<<(unsigned)((n0 + 1 + 255) / 256), 256, 0, stream>>>(c, n0, csf->slice_ptr));
+            CB_CUDA(cudaGetLastError());
+            return csf_rebin(csf, stream);
+        };
+        rc = body();
+    }
+    if (rc != CONST_OK) {
+        csf_free(csf);
+        return rc;
+    }
+    *out = csf;
+    return CONST_OK;
+}
+
+}  // namespace cb

@@ -334,7 +334,7 @@ def network_workload(n=1024, n_k=128, band=32, keep=0.25, *, seed=0, config_id=5
         sparse={"U": U, "W": W}, dense={"V": V},
         expression="Z[i,m] = U[i,j,k] * V[j,l] * W[k,l,m]",
         tree=["T[i,k,l] = U[i,j,k] * V[j,l]", "Z[i,m] = T[i,k,l] * W[k,l,m]"],
-        mode_orders={"U": (0, 1, 2), "W": (0, 1, 2)}, loop_orders=["ijkl", "iklm"],
+        mode_orders={"U": (0, 2, 1), "W": (2, 1, 0)}, loop_orders=["ikjl", "imlk"],
         out_shape=(n, n))
 
 
