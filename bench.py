@@ -175,7 +175,7 @@ def main():
         if rank != 0:
             return 0
         w = make_config(args.config, scale=args.scale, seed=0)
-        auto = {1: 20_000, 2: 1_000_000, 3: 400_000, 4: 4_000_000, 5: 60_000}[args.config]
+        auto = {1: 20_000, 2: 40_000_000, 3: 8_000_000, 4: 100_000_000, 5: 400_000}[args.config]
         target = args.oracle_nnz or auto
         for _ in range(args.warmup):
             time_oracle(w, target)
@@ -372,7 +372,7 @@ def main():
     fused = next((rooflines[k] for k in rooflines if k in fused_names and rooflines[k]), None)
 
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ----
-    auto = {1: 20_000, 2: 1_000_000, 3: 400_000, 4: 4_000_000, 5: 60_000}[args.config]
+    auto = {1: 20_000, 2: 40_000_000, 3: 8_000_000, 4: 100_000_000, 5: 400_000}[args.config]
     cpu_baseline, _ = time_oracle(w, args.oracle_nnz or auto)
 
     line = {
