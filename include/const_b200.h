@@ -75,6 +75,40 @@ const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz,
                                const int32_t *const *coords_dev, const void *vals_dev, const_dtype_t dtype,
                                const int *mode_order, void *stream, const_csf_t **out);
 
+/*
+ * COO -> CSF without any allocation.  (The paper has no counterpart: this exists for deployment.)
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point where it must build a
+ * CSF tensor -- a plug-in running inside a host application that hands out a fixed arena and
+ * forbids cudaMalloc, a real-time loop where the driver's allocation lock and its unbounded latency
+ * are unacceptable, or a process already so close to the memory limit that a temporary allocation
+ * could fail.  const_csf_build cannot serve them, because it obtains its sort buffers, scan
+ * buffers and result arrays from the stream-ordered allocator.
+ *
+ * Same arguments and same result arrays as const_csf_build, except that the caller supplies the
+ * outputs and no handle is created (so there are no work lists: the arrays are the product):
+ *   pos_out_dev[l]  device buffer of at least nnz + 1 int32 (2 for l = 0);
+ *   crd_out_dev[l]  device buffer of at least nnz int32;
+ *   vals_out_dev    device buffer of nnz values of `dtype`; also used as a sort buffer during the call;
+ *   level_sizes     host array of `order` entries (may be NULL): number of nodes of each level.
+ * Every temporary lives in one array that the library holds in static device memory, about 6.4 MB
+ * on every GPU that loads the library, for as long as the process runs.  Limit: nnz <= 262 144;
+ * a larger nnz returns CONST_ERR_WORKSPACE and touches nothing.  The call issues no cudaMalloc,
+ * cudaFree, stream-ordered allocation or allocating library routine.
+ *
+ * The first call on each device looks up the device address of that array (one
+ * cudaGetSymbolAddress with that device current); make that first call outside any stream capture.
+ * All calls share the array and it keeps whatever the previous call left in it; the call clears the
+ * parts that must start at zero.  Two calls whose GPU work overlaps (different streams, or different
+ * host threads) race on it: serialise them.  Like const_csf_build, the call synchronises the stream
+ * once to read the level sizes and the error word, and returns the same error codes.
+ */
+const_status_t const_csf_build_noalloc(int order, const int64_t *dims, int64_t nnz,
+                                       const int32_t *const *coords_dev, const void *vals_dev, const_dtype_t dtype,
+                                       const int *mode_order, void *stream,
+                                       int32_t *const *pos_out_dev, int32_t *const *crd_out_dev, void *vals_out_dev,
+                                       int64_t *level_sizes);
+
 /* Borrowed device pointers of one level (valid until const_destroy).  *pos has n_{level-1}+1 entries
  * (2 for level 0), *crd has *n entries.  Any output pointer may be NULL. */
 const_status_t const_csf_level(const const_csf_t *csf, int level, const int32_t **pos, const int32_t **crd,

@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     F64,
     STATUS_NAMES,
     const_csf_build,
+    const_csf_build_noalloc,
     const_csf_level,
     const_csf_values,
     const_csf_set_bins,

@@ -54,6 +54,9 @@ def load_library():
     vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
     pp = ctypes.POINTER
     lib.const_csf_build.argtypes = [i32, pp(i64), i64, pp(vp), vp, i32, pp(i32), vp, pp(vp)]
+    lib.const_csf_build_noalloc.argtypes = [i32, pp(i64), i64, pp(vp), vp, i32, pp(i32), vp, pp(vp), pp(vp), vp,
+                                            pp(i64)]
+    lib.const_csf_build_noalloc.restype = i32
     lib.const_csf_level.argtypes = [vp, i32, pp(vp), pp(vp), pp(i64)]
     lib.const_csf_values.argtypes = [vp, pp(vp), pp(i64)]
     lib.const_csf_set_bins.argtypes = [vp, i64, i64, i64, vp]
@@ -145,6 +148,39 @@ def const_csf_build(coords, vals, dims: Sequence[int], mode_order: Sequence[int]
                              _stream_ptr(stream), ctypes.byref(out))
     _check(st, "const_csf_build")
     return CsfHandle(out.value, order, dtype)
+
+
+def const_csf_build_noalloc(coords, vals, dims: Sequence[int], mode_order: Sequence[int], pos_out, crd_out,
+                            vals_out, stream=None) -> List[int]:
+    """COO -> CSF into buffers the caller owns, for callers that may not allocate device memory.
+
+    pos_out / crd_out: one int32 CUDA tensor per level with room for nnz + 1 / nnz entries;
+    vals_out: CUDA tensor like `vals`.  Nothing is allocated on the device by this call (the
+    library's temporaries sit in a fixed static array, which limits nnz to 262 144).
+    Returns the number of nodes per level.
+    """
+    import torch
+    lib = load_library()
+    order = len(dims)
+    nnz = int(vals.numel())
+    dtype = F32 if vals.dtype == torch.float32 else F64
+    for l in range(order):
+        if pos_out[l].dtype != torch.int32 or crd_out[l].dtype != torch.int32:
+            raise ValueError("pos/crd outputs must be int32")
+        if pos_out[l].numel() < (2 if l == 0 else nnz + 1) or crd_out[l].numel() < nnz:
+            raise ValueError("output buffer too small")
+    if vals_out.dtype != vals.dtype or vals_out.numel() < nnz:
+        raise ValueError("vals_out must match vals")
+    dims_a = (ctypes.c_int64 * order)(*[int(d) for d in dims])
+    mo_a = (ctypes.c_int * order)(*[int(m) for m in mode_order])
+    cptr = (ctypes.c_void_p * order)(*[c.data_ptr() for c in coords])
+    pptr = (ctypes.c_void_p * order)(*[p.data_ptr() for p in pos_out])
+    rptr = (ctypes.c_void_p * order)(*[c.data_ptr() for c in crd_out])
+    sizes = (ctypes.c_int64 * order)()
+    st = lib.const_csf_build_noalloc(order, dims_a, nnz, cptr, ctypes.c_void_p(vals.data_ptr()), dtype, mo_a,
+                                     _stream_ptr(stream), pptr, rptr, ctypes.c_void_p(vals_out.data_ptr()), sizes)
+    _check(st, "const_csf_build_noalloc")
+    return list(sizes)
 
 
 def _dev_to_torch(ptr: Optional[int], n: int, dtype):

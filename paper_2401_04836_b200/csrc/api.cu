@@ -64,6 +64,24 @@ const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz, cons
     return rc;
 }
 
+const_status_t const_csf_build_noalloc(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
+                                       const void *vals_dev, const_dtype_t dtype, const int *mode_order, void *stream,
+                                       int32_t *const *pos_out_dev, int32_t *const *crd_out_dev, void *vals_out_dev,
+                                       int64_t *level_sizes) {
+    if (order < 2 || order > kMaxOrder || !dims || nnz < 0 || !coords_dev || !mode_order || !pos_out_dev ||
+        !crd_out_dev || (dtype != CONST_F32 && dtype != CONST_F64) || (nnz > 0 && (!vals_dev || !vals_out_dev)))
+        return CONST_ERR_INVALID_ARG;
+    bool seen[kMaxOrder] = {false, false, false, false};
+    for (int l = 0; l < order; ++l) {
+        if (mode_order[l] < 0 || mode_order[l] >= order || seen[mode_order[l]]) return CONST_ERR_INVALID_ARG;
+        seen[mode_order[l]] = true;
+        if (dims[l] < 1 || !pos_out_dev[l] || (nnz > 0 && (!coords_dev[l] || !crd_out_dev[l]))) return CONST_ERR_INVALID_ARG;
+    }
+    return csf_build_noalloc_impl(order, dims, nnz, coords_dev, vals_dev, dtype, mode_order,
+                                  static_cast<cudaStream_t>(stream), pos_out_dev, crd_out_dev, vals_out_dev,
+                                  level_sizes);
+}
+
 const_status_t const_csf_level(const const_csf_t *h, int level, const int32_t **pos, const int32_t **crd, int64_t *n) {
     const const_csf *c = as_csf(h);
     if (!c || level < 0 || level >= c->order) return CONST_ERR_INVALID_ARG;

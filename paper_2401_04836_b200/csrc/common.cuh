@@ -91,6 +91,10 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
                               cudaStream_t stream, const_csf **out);
 const_status_t csf_rebin(const_csf *csf, cudaStream_t stream);
 void csf_free(const_csf *csf);
+const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
+                                      const void *vals_dev, const_dtype_t dtype, const int *mode_order,
+                                      cudaStream_t stream, int32_t *const *pos_out, int32_t *const *crd_out,
+                                      void *vals_out, int64_t *level_sizes);
 
 // chain_kernels.cu
 const_status_t run_ttmc3(const const_csf *X, const float *U, const float *V, int R2, int R3, float *Y,

@@ -721,4 +721,151 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
     return CONST_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// const_csf_build_noalloc: the same COO -> CSF pipeline with every temporary in one static device
+// array, for callers that must not allocate (see include/const_b200.h).
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t kNoAllocMaxNnz = 1 << 18;                               // 262 144 nonzeros
+constexpr size_t kNaKeys = sizeof(uint64_t) * kNoAllocMaxNnz;             // one key buffer / one fp64 payload buffer
+constexpr size_t kNaTiles = (kNoAllocMaxNnz + kRsTile - 1) / kRsTile;
+constexpr size_t kNaCpBlocks = (kNoAllocMaxNnz + kCpTile - 1) / kCpTile;
+// byte offsets inside the static array (every region 256-byte aligned)
+constexpr size_t kNaOffKeys0 = 0;
+constexpr size_t kNaOffKeys1 = kNaOffKeys0 + kNaKeys;
+constexpr size_t kNaOffVals = kNaOffKeys1 + kNaKeys;                      // second payload buffer (the first is the caller's output)
+constexpr size_t kNaOffTileStatus = kNaOffVals + kNaKeys;
+constexpr size_t kNaOffHist = kNaOffTileStatus + sizeof(unsigned long long) * kNaTiles * kRsBins;
+constexpr size_t kNaOffBlockCounts = kNaOffHist + sizeof(uint32_t) * kMaxPasses * kRsBins;
+constexpr size_t kNaOffSmall = kNaOffBlockCounts + ((sizeof(uint32_t) * kCpLevels * kNaCpBlocks + 255) / 256) * 256;
+constexpr size_t kNaSmallBytes = 256;                                     // pass counters [8], level totals [4], status word
+constexpr size_t kNaBytes = kNaOffSmall + kNaSmallBytes;
+
+// The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress: it is not
+// a device address and must never be handed to a kernel or to cudaMemset as if it were one.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
+
+constexpr int kNaMaxDevices = 64;
+unsigned char *g_noalloc_ptr[kNaMaxDevices] = {nullptr};                  // device address of the array, per device
+
+const_status_t noalloc_scratch(unsigned char **out) {
+    int dev = 0;
+    CB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kNaMaxDevices) return CONST_ERR_UNSUPPORTED;
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        CB_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));                 // resolved with `dev` current
+        g_noalloc_ptr[dev] = static_cast<unsigned char *>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return CONST_OK;
+}
+
+template <typename V>
+const_status_t noalloc_sort(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
+                            unsigned char *base, int32_t *status, cudaStream_t stream) {
+    uint32_t *hist = reinterpret_cast<uint32_t *>(base + kNaOffHist);
+    uint32_t *counters = reinterpret_cast<uint32_t *>(base + kNaOffSmall);
+    unsigned long long *tile_status = reinterpret_cast<unsigned long long *>(base + kNaOffTileStatus);
+    const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
+    int hist_blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    rs_histogram<<<hist_blocks, 256, 0, stream>>>(keys, n, passes, hist);
+    rs_scan_hist<<<passes, 256, 0, stream>>>(hist);
+    const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
+    CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    for (int p = 0; p < passes; ++p) {
+        CB_CUDA(cudaMemsetAsync(tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
+        rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(keys, keys_alt, vals, vals_alt, n, 8 * p,
+                                                                     hist + p * kRsBins, tile_status, counters + p, status);
+        std::swap(keys, keys_alt);
+        std::swap(vals, vals_alt);
+    }
+    CB_CUDA(cudaGetLastError());
+    return CONST_OK;
+}
+
+}  // namespace
+
+const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
+                                      const void *vals_dev, const_dtype_t dtype, const int *mode_order,
+                                      cudaStream_t stream, int32_t *const *pos_out, int32_t *const *crd_out,
+                                      void *vals_out, int64_t *level_sizes) {
+    if (nnz > kNoAllocMaxNnz) return CONST_ERR_WORKSPACE;
+    int bits[kMaxOrder] = {0, 0, 0, 0}, shift[kMaxOrder] = {0, 0, 0, 0};
+    int total_bits = 0;
+    for (int l = 0; l < order; ++l) { bits[l] = bits_for(dims[mode_order[l]]); total_bits += bits[l]; }
+    if (total_bits > 64) return CONST_ERR_UNSUPPORTED;
+    int acc = 0;
+    for (int l = order - 1; l >= 0; --l) { shift[l] = acc; acc += bits[l]; }
+    const int passes = (total_bits + 7) / 8;
+
+    unsigned char *base = nullptr;
+    const_status_t rc = noalloc_scratch(&base);
+    if (rc != CONST_OK) return rc;
+    uint64_t *keys = reinterpret_cast<uint64_t *>(base + kNaOffKeys0);
+    uint64_t *keys_alt = reinterpret_cast<uint64_t *>(base + kNaOffKeys1);
+    uint32_t *block_counts = reinterpret_cast<uint32_t *>(base + kNaOffBlockCounts);
+    uint32_t *totals = reinterpret_cast<uint32_t *>(base + kNaOffSmall + 64);
+    int32_t *status = reinterpret_cast<int32_t *>(base + kNaOffSmall + 128);
+    // everything that must start at zero: digit histograms, pass counters, level totals, status word
+    CB_CUDA(cudaMemsetAsync(base + kNaOffHist, 0, sizeof(uint32_t) * kMaxPasses * kRsBins, stream));
+    CB_CUDA(cudaMemsetAsync(base + kNaOffSmall, 0, kNaSmallBytes, stream));
+
+    const size_t vsize = dtype == CONST_F32 ? 4 : 8;
+    const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
+    LevelShifts ls;
+    ls.order = order;
+    for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = shift[l];
+    if (nnz > 0) {
+        PackArgs pa;
+        pa.order = order;
+        for (int l = 0; l < kMaxOrder; ++l) {
+            pa.c[l] = l < order ? coords_dev[mode_order[l]] : nullptr;
+            pa.dim[l] = l < order ? dims[mode_order[l]] : 0;
+            pa.shift[l] = shift[l];
+        }
+        pack_keys<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(pa, nnz, keys, status);
+        // the payload ping-pongs between the caller's output and the static buffer; start on the side
+        // that makes the last pass land in the caller's output
+        void *va = vals_out, *vb = base + kNaOffVals;
+        void *first = (passes % 2 == 0) ? va : vb, *second = (passes % 2 == 0) ? vb : va;
+        CB_CUDA(cudaMemcpyAsync(first, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
+        if (dtype == CONST_F32) {
+            uint32_t *v = (uint32_t *)first, *w = (uint32_t *)second;
+            rc = noalloc_sort<uint32_t>(keys, keys_alt, v, w, nnz, passes, base, status, stream);
+        } else {
+            unsigned long long *v = (unsigned long long *)first, *w = (unsigned long long *)second;
+            rc = noalloc_sort<unsigned long long>(keys, keys_alt, v, w, nnz, passes, base, status, stream);
+        }
+        if (rc != CONST_OK) return rc;
+        csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status);
+        csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals);
+    }
+    uint32_t h_totals[4] = {0, 0, 0, 0};
+    int32_t h_status = 0;
+    CB_CUDA(cudaMemcpyAsync(h_totals, totals, sizeof(h_totals), cudaMemcpyDeviceToHost, stream));
+    CB_CUDA(cudaMemcpyAsync(&h_status, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    CB_CUDA(cudaStreamSynchronize(stream));
+    if (h_status != 0) return (const_status_t)h_status;
+    LevelSizes sz;
+    sz.order = order;
+    for (int l = 0; l < kMaxOrder; ++l) sz.n[l] = 0;
+    for (int l = 0; l < order - 1; ++l) sz.n[l] = h_totals[l];
+    sz.n[order - 1] = nnz;
+    CsfArrays arr;
+    for (int l = 0; l < kMaxOrder; ++l) {
+        arr.pos[l] = l < order ? pos_out[l] : nullptr;
+        arr.crd[l] = l < order ? crd_out[l] : nullptr;
+        arr.bits[l] = bits[l];
+    }
+    if (nnz > 0) csf_scatter<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, arr);
+    csf_finish<<<1, 32, 0, stream>>>(arr, sz);
+    CB_CUDA(cudaGetLastError());
+    if (level_sizes)
+        for (int l = 0; l < order; ++l) level_sizes[l] = sz.n[l];
+    return CONST_OK;
+}
+
 }  // namespace cb
