@@ -35,59 +35,58 @@ enum DevErr : int32_t { kErrNone = 0 };
 
 __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicCAS(status, 0, code); }
 
-__global__ void pack_keys(PackArgs a, int64_t nnz, uint64_t *__restrict__ keys, int32_t *status) {
-    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= nnz) return;
-    uint64_t key = 0;
+constexpr int kRsBins = 256;
+constexpr int kMaxPasses = 8;
+
+// Pack the permuted coordinates of every nonzero into its 64-bit sort key (range-checked) and, in the
+// same read, count the 8-bit digits of every radix pass.  Per-block counts live in shared memory and
+// are flushed once; the grid is sized to a few blocks per SM so the flush stays small.
+template <int ORDER>
+__global__ void __launch_bounds__(256) pack_hist(PackArgs a, int64_t nnz, int passes, uint64_t *__restrict__ keys,
+                                                 uint32_t *__restrict__ hist, int32_t *status) {
+    __shared__ uint32_t sh[kMaxPasses * kRsBins];
+    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x) sh[x] = 0;
+    __syncthreads();
     bool bad = false;
-    for (int l = 0; l < a.order; ++l) {
-        int64_t c = a.c[l][e];
-        if (c < 0 || c >= a.dim[l]) { bad = true; c = 0; }
-        key |= (uint64_t)c << a.shift[l];
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < nnz; e += stride) {
+        uint64_t key = 0;
+#pragma unroll
+        for (int l = 0; l < ORDER; ++l) {
+            int64_t c = __ldg(a.c[l] + e);
+            if (c < 0 || c >= a.dim[l]) { bad = true; c = 0; }
+            key |= (uint64_t)c << a.shift[l];
+        }
+        keys[e] = key;
+        for (int p = 0; p < passes; ++p) atomicAdd(&sh[p * kRsBins + ((unsigned)(key >> (8 * p)) & 255u)], 1u);
     }
     if (bad) report(status, CONST_ERR_COORD_RANGE);
-    keys[e] = key;
+    __syncthreads();
+    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x)
+        if (sh[x]) atomicAdd(&hist[x], sh[x]);
+}
+
+inline void launch_pack_hist(const PackArgs &pa, int64_t nnz, int passes, uint64_t *keys, uint32_t *hist,
+                             int32_t *status, cudaStream_t stream) {
+    const int blocks = (int)std::min<int64_t>((nnz + 255) / 256, 148 * 8);
+    switch (pa.order) {
+        case 2: pack_hist<2><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
+        case 3: pack_hist<3><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
+        default: pack_hist<4><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
 // radix sort
 // ------------------------------------------------------------------------------------------------
-constexpr int kRsBins = 256;
 constexpr int kRsThreads = 256;
 constexpr int kRsItems = 16;
 constexpr int kRsTile = kRsThreads * kRsItems;     // 4096 keys per tile
 constexpr int kRsWarps = kRsThreads / 32;
-constexpr int kMaxPasses = 8;
 constexpr uint64_t kFlagAgg = 1ull << 62;          // tile published its own digit counts
 constexpr uint64_t kFlagInc = 2ull << 62;          // tile published counts summed over all earlier tiles too
-constexpr uint64_t kValMask = (1ull << 62) - 1;
+constexpr uint64_t kValMask = (1ull << 32) - 1;       // low 32 bits: count; bits 32..39: pass number + 1
 constexpr int kSpinLimit = 1 << 21;
-
-// Digit histograms of every pass in one read of the keys.
-__global__ void __launch_bounds__(256) rs_histogram(const uint64_t *__restrict__ keys, int64_t n, int passes,
-                                                    uint32_t *__restrict__ hist) {
-    __shared__ uint32_t sh[kMaxPasses * kRsBins];
-    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x) sh[x] = 0;
-    __syncthreads();
-    const int lane = threadIdx.x & 31;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t base = (int64_t)blockIdx.x * blockDim.x; base < n; base += stride) {   // base is block-uniform
-        int64_t e = base + threadIdx.x;
-        bool valid = e < n;
-        unsigned active = __ballot_sync(0xffffffffu, valid);
-        if (valid) {
-            uint64_t key = keys[e];
-            for (int p = 0; p < passes; ++p) {
-                unsigned d = (unsigned)(key >> (8 * p)) & 255u;
-                unsigned peers = __match_any_sync(active, d);
-                if (lane == __ffs(peers) - 1) atomicAdd(&sh[p * kRsBins + d], __popc(peers));
-            }
-        }
-    }
-    __syncthreads();
-    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x)
-        if (sh[x]) atomicAdd(&hist[x], sh[x]);
-}
 
 // Exclusive scan of each pass's 256-bin histogram: one block per pass.
 __global__ void __launch_bounds__(256) rs_scan_hist(uint32_t *hist) {
@@ -108,7 +107,7 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
                                                          const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
                                                          int shift, const uint32_t *__restrict__ digit_base,
                                                          unsigned long long *status, uint32_t *counter,
-                                                         int32_t *err) {
+                                                         int32_t *err, unsigned epoch) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t *keybuf = reinterpret_cast<uint64_t *>(smem_raw);
     V *valbuf = reinterpret_cast<V *>(smem_raw + kRsTile * sizeof(uint64_t));
@@ -178,7 +177,10 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
 
     // chained scan over tiles (decoupled look-back); every wait is bounded
     volatile unsigned long long *st = status;
-    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | (unsigned long long)count;
+    // A status word counts only if it carries this pass's number, so the array is cleared once per
+    // sort, not once per pass.
+    const unsigned long long tag = (unsigned long long)epoch << 32;
+    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | tag | (unsigned long long)count;
     unsigned long long before = 0;
     if (tile > 0) {
         bool ok = true;
@@ -188,7 +190,7 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
             int spins = 0;
             for (;;) {
                 s = st[t * kRsBins + d];
-                if (s >> 62) break;
+                if ((s >> 62) && ((s >> 32) & 0xffu) == epoch) break;
                 if (++spins > kSpinLimit) { ok = false; break; }
                 if (spins > 64) __nanosleep(100);
             }
@@ -198,7 +200,7 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
             --t;
         }
         if (ok) {
-            st[tile * kRsBins + d] = kFlagInc | (before + count);
+            st[tile * kRsBins + d] = kFlagInc | tag | (before + count);
         } else {
             report(err, CONST_ERR_TIMEOUT);
             s_abort = 1;
@@ -454,37 +456,49 @@ __global__ void __launch_bounds__(1024) bin_scan(const int32_t *__restrict__ sli
 }
 
 __global__ void bin_fill(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t light_max,
-                         int64_t heavy_max, int64_t chunk, const int32_t *__restrict__ item_off,
+                         int64_t heavy_max, const int32_t *__restrict__ item_off,
                          const int32_t *__restrict__ light_idx, WorkItem *__restrict__ items,
                          int32_t *__restrict__ light_list) {
     int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n0) return;
+    const int64_t z = (int64_t)slice_ptr[s + 1] - slice_ptr[s];
+    if (z <= light_max) light_list[light_idx[s]] = (int32_t)s;
+    else if (z <= heavy_max) items[item_off[s]] = WorkItem{(int32_t)s, c.pos[1][s], c.pos[1][s + 1], kItemBlock};
+}
+
+// One thread per block work item of the heavy/giant range: items of giant slices find their own
+// level-1 node range (the slice is cut where the leaf offset passes q/parts of its nonzeros).
+__global__ void bin_fill_chunks(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t heavy_max,
+                                int64_t chunk, const int32_t *__restrict__ item_off, int64_t n_hg_items,
+                                WorkItem *__restrict__ items) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_hg_items) return;
+    // slice owning item t: last s with item_off[s] <= t (slices without items share their successor's offset)
+    int64_t lo = 0, hi = n0 - 1;
+    while (lo < hi) {
+        int64_t mid = lo + (hi - lo + 1) / 2;
+        if (item_off[mid] <= t) lo = mid; else hi = mid - 1;
+    }
+    const int64_t s = lo;
     const int32_t p0 = slice_ptr[s], p1 = slice_ptr[s + 1];
     const int64_t z = (int64_t)p1 - p0;
+    if (z <= heavy_max) return;                       // a whole-slice item, written by bin_fill
+    const int64_t parts = (z + chunk - 1) / chunk, q = t - item_off[s];
     const int32_t f0 = c.pos[1][s], f1 = c.pos[1][s + 1];
-    if (z <= light_max) {
-        light_list[light_idx[s]] = (int32_t)s;
-    } else if (z <= heavy_max) {
-        items[item_off[s]] = WorkItem{(int32_t)s, f0, f1, kItemBlock};
-    } else {
-        const int64_t parts = (z + chunk - 1) / chunk;
-        int32_t begin = f0;
-        for (int64_t q = 0; q < parts; ++q) {
-            int32_t end = f1;
-            if (q + 1 < parts) {
-                // first level-1 node whose leaf offset reaches the target
-                const int64_t target = p0 + (z * (q + 1)) / parts;
-                int32_t lo = begin, hi = f1;
-                while (lo < hi) {
-                    int32_t mid = lo + (hi - lo) / 2;
-                    if ((int64_t)leaf_of_fiber(c, mid) < target) lo = mid + 1; else hi = mid;
-                }
-                end = lo;
-            }
-            items[item_off[s] + q] = WorkItem{(int32_t)s, begin, end, kItemChunk};
-            begin = end;
+    int32_t cut[2];
+    for (int e = 0; e < 2; ++e) {
+        const int64_t qq = q + e;
+        if (qq == 0) { cut[e] = f0; continue; }
+        if (qq >= parts) { cut[e] = f1; continue; }
+        const int64_t target = p0 + (z * qq) / parts;
+        int32_t a = f0, b = f1;
+        while (a < b) {
+            int32_t mid = a + (b - a) / 2;
+            if ((int64_t)leaf_of_fiber(c, mid) < target) a = mid + 1; else b = mid;
         }
+        cut[e] = a;
     }
+    items[t] = WorkItem{(int32_t)s, cut[0], cut[1], kItemChunk};
 }
 
 __global__ void bin_light_items(WorkItem *__restrict__ items, int64_t first_item, int64_t n_light) {
@@ -502,13 +516,43 @@ int bits_for(int64_t extent) {
     return b;
 }
 
+// Stream-ordered memory comes from a pool the library owns (one per device) whose release threshold
+// is unlimited, so buffers freed by one build are reused by the next without going back to the driver.
+cudaMemPool_t library_pool(int device) {
+    static cudaMemPool_t pools[64] = {nullptr};
+    if (device < 0 || device >= 64) return nullptr;
+    if (!pools[device]) {
+        cudaMemPoolProps props;
+        std::memset(&props, 0, sizeof(props));
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        cudaMemPool_t pool = nullptr;
+        if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) return nullptr;
+        unsigned long long keep = ~0ull;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        pools[device] = pool;
+    }
+    return pools[device];
+}
+
+cudaError_t pool_alloc(void **p, size_t bytes, cudaStream_t stream) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    cudaMemPool_t pool = library_pool(dev);
+    if (!pool) return cudaMallocAsync(p, bytes ? bytes : 16, stream);
+    return cudaMallocFromPoolAsync(p, bytes ? bytes : 16, pool, stream);
+}
+
 struct Scratch {            // stream-ordered temporaries of one build
     cudaStream_t stream;
     void *ptrs[16];
     int n = 0;
     explicit Scratch(cudaStream_t s) : stream(s) {}
     cudaError_t alloc(void **p, size_t bytes) {
-        cudaError_t e = cudaMallocAsync(p, bytes ? bytes : 16, stream);
+        cudaError_t e = pool_alloc(p, bytes, stream);
         if (e == cudaSuccess) ptrs[n++] = *p;
         return e;
     }
@@ -520,33 +564,85 @@ struct Scratch {            // stream-ordered temporaries of one build
     }
 };
 
+// Small buffers of one sort.  `zeroed` covers hist, counters, totals and the status word in one
+// allocation so that a single memset clears them.
+struct SortBufs {
+    uint32_t *hist;                    // [kMaxPasses][256] digit counts, then exclusive digit offsets
+    uint32_t *counters;                // [kMaxPasses] tile tickets
+    unsigned long long *tile_status;   // [ntiles][256]
+};
+
 template <typename V>
-const_status_t sort_pairs(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
-                          Scratch &tmp, int32_t *status, cudaStream_t stream) {
+const_status_t sort_passes(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
+                           const SortBufs &b, int32_t *status, cudaStream_t stream) {
     if (n == 0 || passes == 0) return CONST_OK;
-    uint32_t *hist = nullptr, *counters = nullptr;
-    unsigned long long *tile_status = nullptr;
     const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
-    CB_CUDA(tmp.alloc((void **)&hist, sizeof(uint32_t) * kMaxPasses * kRsBins));
-    CB_CUDA(tmp.alloc((void **)&counters, sizeof(uint32_t) * kMaxPasses));
-    CB_CUDA(tmp.alloc((void **)&tile_status, sizeof(unsigned long long) * ntiles * kRsBins));
-    CB_CUDA(cudaMemsetAsync(hist, 0, sizeof(uint32_t) * kMaxPasses * kRsBins, stream));
-    CB_CUDA(cudaMemsetAsync(counters, 0, sizeof(uint32_t) * kMaxPasses, stream));
-    int hist_blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
-    CB_LAUNCH("rs_histogram", stream, rs_histogram<<<hist_blocks, 256, 0, stream>>>(keys, n, passes, hist));
-    CB_LAUNCH("rs_scan_hist", stream, rs_scan_hist<<<passes, 256, 0, stream>>>(hist));
+    CB_CUDA(cudaMemsetAsync(b.tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
+    CB_LAUNCH("rs_scan_hist", stream, rs_scan_hist<<<passes, 256, 0, stream>>>(b.hist));
     const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
-    CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    static bool attr_set[64] = {false};    // per template instance and device
+    int dev = 0;
+    CB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
     for (int p = 0; p < passes; ++p) {
-        CB_CUDA(cudaMemsetAsync(tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
-        CB_LAUNCH("rs_onesweep", stream, rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(keys, keys_alt, vals, vals_alt, n, 8 * p,
-                                                                     hist + p * kRsBins, tile_status, counters + p,
-                                                                     status));
+        CB_LAUNCH("rs_onesweep", stream,
+                  rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(
+                      keys, keys_alt, vals, vals_alt, n, 8 * p, b.hist + p * kRsBins, b.tile_status, b.counters + p,
+                      status, (unsigned)(p + 1)));
         std::swap(keys, keys_alt);
         std::swap(vals, vals_alt);
     }
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
+}
+
+// Everything between "keys packed" and "level sizes known": sort, flag counts, block scan.
+const_status_t sort_and_count(uint64_t *&keys, uint64_t *&keys_alt, void *&vals, void *&vals_alt, int64_t nnz,
+                              int passes, const_dtype_t dtype, const SortBufs &b, const LevelShifts &ls,
+                              uint32_t *block_counts, uint32_t *totals, int32_t *status, cudaStream_t stream) {
+    const_status_t s;
+    if (dtype == CONST_F32) {
+        uint32_t *v = (uint32_t *)vals, *va = (uint32_t *)vals_alt;
+        s = sort_passes<uint32_t>(keys, keys_alt, v, va, nnz, passes, b, status, stream);
+        vals = v; vals_alt = va;
+    } else {
+        unsigned long long *v = (unsigned long long *)vals, *va = (unsigned long long *)vals_alt;
+        s = sort_passes<unsigned long long>(keys, keys_alt, v, va, nnz, passes, b, status, stream);
+        vals = v; vals_alt = va;
+    }
+    if (s != CONST_OK) return s;
+    const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
+    CB_LAUNCH("csf_count", stream, csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status));
+    CB_LAUNCH("csf_scan_blocks", stream, csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals));
+    return CONST_OK;
+}
+
+struct KeyLayout { int bits[kMaxOrder]; int shift[kMaxOrder]; int total_bits; int passes; };
+
+bool key_layout(int order, const int64_t *dims, const int *mode_order, KeyLayout &k) {
+    k.total_bits = 0;
+    for (int l = 0; l < kMaxOrder; ++l) k.bits[l] = k.shift[l] = 0;
+    for (int l = 0; l < order; ++l) { k.bits[l] = bits_for(dims[mode_order[l]]); k.total_bits += k.bits[l]; }
+    if (k.total_bits > 64) return false;
+    int acc = 0;
+    for (int l = order - 1; l >= 0; --l) { k.shift[l] = acc; acc += k.bits[l]; }
+    k.passes = (k.total_bits + 7) / 8;
+    return true;
+}
+
+PackArgs pack_args(int order, const int64_t *dims, const int *mode_order, const int32_t *const *coords_dev,
+                   const KeyLayout &k) {
+    PackArgs pa;
+    pa.order = order;
+    for (int l = 0; l < kMaxOrder; ++l) {
+        pa.c[l] = l < order ? coords_dev[mode_order[l]] : nullptr;
+        pa.dim[l] = l < order ? dims[mode_order[l]] : 0;
+        pa.shift[l] = k.shift[l];
+    }
+    return pa;
 }
 
 }  // namespace
@@ -592,11 +688,13 @@ const_status_t csf_rebin(const_csf *csf, cudaStream_t stream) {
     csf->n_giant = h[3];
     const int64_t light_groups = (csf->n_light + kWarpsPerBlock - 1) / kWarpsPerBlock;
     csf->n_items = hg_items + light_groups;
-    CB_CUDA(cudaMallocAsync((void **)&csf->items, sizeof(WorkItem) * std::max<int64_t>(csf->n_items, 1), stream));
-    CB_CUDA(cudaMallocAsync((void **)&csf->light_list, sizeof(int32_t) * std::max<int64_t>(csf->n_light, 1), stream));
+    CB_CUDA(pool_alloc((void **)&csf->items, sizeof(WorkItem) * std::max<int64_t>(csf->n_items, 1), stream));
+    CB_CUDA(pool_alloc((void **)&csf->light_list, sizeof(int32_t) * std::max<int64_t>(csf->n_light, 1), stream));
     CB_LAUNCH("bin_fill", stream, bin_fill<<<(unsigned)((n0 + 255) / 256), 256, 0, stream>>>(c, csf->slice_ptr, n0, csf->light_max, csf->heavy_max,
-                                                              csf->chunk, item_off, light_idx, csf->items,
-                                                              csf->light_list));
+                                                              item_off, light_idx, csf->items, csf->light_list));
+    if (hg_items > 0)
+        CB_LAUNCH("bin_fill_chunks", stream, bin_fill_chunks<<<(unsigned)((hg_items + 127) / 128), 128, 0, stream>>>(
+                      c, csf->slice_ptr, n0, csf->heavy_max, csf->chunk, item_off, hg_items, csf->items));
     if (light_groups > 0)
         CB_LAUNCH("bin_light_items", stream, bin_light_items<<<(unsigned)((light_groups + 255) / 256), 256, 0, stream>>>(csf->items, hg_items, csf->n_light));
     CB_CUDA(cudaGetLastError());
@@ -606,14 +704,8 @@ const_status_t csf_rebin(const_csf *csf, cudaStream_t stream) {
 const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
                               const void *vals_dev, const_dtype_t dtype, const int *mode_order,
                               cudaStream_t stream, const_csf **out) {
-    // level layout of the packed key
-    int bits[kMaxOrder] = {0, 0, 0, 0}, shift[kMaxOrder] = {0, 0, 0, 0};
-    int total_bits = 0;
-    for (int l = 0; l < order; ++l) { bits[l] = bits_for(dims[mode_order[l]]); total_bits += bits[l]; }
-    if (total_bits > 64) return CONST_ERR_UNSUPPORTED;
-    int acc = 0;
-    for (int l = order - 1; l >= 0; --l) { shift[l] = acc; acc += bits[l]; }
-    const int passes = (total_bits + 7) / 8;
+    KeyLayout kl;
+    if (!key_layout(order, dims, mode_order, kl)) return CONST_ERR_UNSUPPORTED;
 
     const_csf *csf = new (std::nothrow) const_csf();
     if (!csf) return CONST_ERR_INVALID_ARG;
@@ -633,61 +725,50 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
         Scratch tmp(stream);
         uint64_t *keys = nullptr, *keys_alt = nullptr;
         void *vals = nullptr, *vals_alt = nullptr;
-        int32_t *status = nullptr;
-        uint32_t *block_counts = nullptr, *totals = nullptr;
+        unsigned char *small = nullptr;          // hist | counters | totals | status, cleared together
+        uint32_t *block_counts = nullptr;
+        SortBufs sb{nullptr, nullptr, nullptr};
         const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
+        const int64_t ntiles = (nnz + kRsTile - 1) / kRsTile;
+        constexpr size_t kHistBytes = sizeof(uint32_t) * kMaxPasses * kRsBins;
+        constexpr size_t kSmallBytes = kHistBytes + 256;
         auto body = [&]() -> const_status_t {
             CB_CUDA(tmp.alloc((void **)&keys, sizeof(uint64_t) * nnz));
             CB_CUDA(tmp.alloc((void **)&keys_alt, sizeof(uint64_t) * nnz));
             CB_CUDA(tmp.alloc(&vals, vsize * nnz));
             CB_CUDA(tmp.alloc(&vals_alt, vsize * nnz));
-            CB_CUDA(tmp.alloc((void **)&status, sizeof(int32_t)));
+            CB_CUDA(tmp.alloc((void **)&small, kSmallBytes));
+            CB_CUDA(tmp.alloc((void **)&sb.tile_status, sizeof(unsigned long long) * std::max<int64_t>(ntiles, 1) * kRsBins));
             CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * kCpLevels * std::max<int64_t>(cp_blocks, 1)));
-            CB_CUDA(tmp.alloc((void **)&totals, sizeof(uint32_t) * 4));
-            CB_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
-            CB_CUDA(cudaMemsetAsync(totals, 0, sizeof(uint32_t) * 4, stream));
+            CB_CUDA(cudaMemsetAsync(small, 0, kSmallBytes, stream));
+            sb.hist = reinterpret_cast<uint32_t *>(small);
+            sb.counters = reinterpret_cast<uint32_t *>(small + kHistBytes);
+            uint32_t *totals = reinterpret_cast<uint32_t *>(small + kHistBytes + 64);
+            int32_t *status = reinterpret_cast<int32_t *>(small + kHistBytes + 128);
             LevelShifts ls;
             ls.order = order;
-            for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = shift[l];
+            for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = kl.shift[l];
             if (nnz > 0) {
-                PackArgs pa;
-                pa.order = order;
-                for (int l = 0; l < kMaxOrder; ++l) {
-                    pa.c[l] = l < order ? coords_dev[mode_order[l]] : nullptr;
-                    pa.dim[l] = l < order ? dims[mode_order[l]] : 0;
-                    pa.shift[l] = shift[l];
-                }
-                CB_LAUNCH("pack_keys", stream, pack_keys<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(pa, nnz, keys, status));
+                PackArgs pa = pack_args(order, dims, mode_order, coords_dev, kl);
+                CB_LAUNCH("pack_hist", stream, launch_pack_hist(pa, nnz, kl.passes, keys, sb.hist, status, stream));
                 CB_CUDA(cudaMemcpyAsync(vals, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
-                const_status_t s;
-                if (dtype == CONST_F32) {
-                    uint32_t *v = (uint32_t *)vals, *va = (uint32_t *)vals_alt;
-                    s = sort_pairs<uint32_t>(keys, keys_alt, v, va, nnz, passes, tmp, status, stream);
-                    vals = v; vals_alt = va;
-                } else {
-                    unsigned long long *v = (unsigned long long *)vals, *va = (unsigned long long *)vals_alt;
-                    s = sort_pairs<unsigned long long>(keys, keys_alt, v, va, nnz, passes, tmp, status, stream);
-                    vals = v; vals_alt = va;
-                }
+                const_status_t s = sort_and_count(keys, keys_alt, vals, vals_alt, nnz, kl.passes, dtype, sb, ls,
+                                                  block_counts, totals, status, stream);
                 if (s != CONST_OK) return s;
-                CB_LAUNCH("csf_count", stream, csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status));
-                CB_LAUNCH("csf_scan_blocks", stream, csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals));
             }
-            uint32_t h_totals[4] = {0, 0, 0, 0};
-            int32_t h_status = 0;
-            CB_CUDA(cudaMemcpyAsync(h_totals, totals, sizeof(h_totals), cudaMemcpyDeviceToHost, stream));
-            CB_CUDA(cudaMemcpyAsync(&h_status, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+            uint32_t h_small[32] = {0};          // totals at [0..4), status at [16]
+            CB_CUDA(cudaMemcpyAsync(h_small, totals, sizeof(uint32_t) * 17, cudaMemcpyDeviceToHost, stream));
             CB_CUDA(cudaStreamSynchronize(stream));
-            if (h_status != 0) return (const_status_t)h_status;
-            for (int l = 0; l < order - 1; ++l) csf->n[l] = h_totals[l];
+            if (h_small[16] != 0) return (const_status_t)h_small[16];
+            for (int l = 0; l < order - 1; ++l) csf->n[l] = h_small[l];
             csf->n[order - 1] = nnz;
 
             CsfArrays arr;
-            for (int l = 0; l < kMaxOrder; ++l) { arr.pos[l] = arr.crd[l] = nullptr; arr.bits[l] = bits[l]; }
+            for (int l = 0; l < kMaxOrder; ++l) { arr.pos[l] = arr.crd[l] = nullptr; arr.bits[l] = kl.bits[l]; }
             for (int l = 0; l < order; ++l) {
                 const int64_t parents = l == 0 ? 1 : csf->n[l - 1];
-                CB_CUDA(cudaMallocAsync((void **)&csf->pos[l], sizeof(int32_t) * (parents + 1), stream));
-                CB_CUDA(cudaMallocAsync((void **)&csf->crd[l], sizeof(int32_t) * std::max<int64_t>(csf->n[l], 1), stream));
+                CB_CUDA(pool_alloc((void **)&csf->pos[l], sizeof(int32_t) * (parents + 1), stream));
+                CB_CUDA(pool_alloc((void **)&csf->crd[l], sizeof(int32_t) * std::max<int64_t>(csf->n[l], 1), stream));
                 arr.pos[l] = csf->pos[l];
                 arr.crd[l] = csf->crd[l];
             }
@@ -702,8 +783,8 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
 
             // per-slice leaf offsets and the default work lists
             const int64_t n0 = csf->n[0];
-            CB_CUDA(cudaMallocAsync((void **)&csf->slice_ptr, sizeof(int32_t) * (n0 + 1), stream));
-            CB_CUDA(cudaMallocAsync((void **)&csf->bin_scratch, sizeof(int32_t) * (2 * (n0 + 1) + 8), stream));
+            CB_CUDA(pool_alloc((void **)&csf->slice_ptr, sizeof(int32_t) * (n0 + 1), stream));
+            CB_CUDA(pool_alloc((void **)&csf->bin_scratch, sizeof(int32_t) * (2 * (n0 + 1) + 8), stream));
             ChainPtrs c;
             c.order = order;
             for (int l = 0; l < kMaxOrder; ++l) c.pos[l] = csf->pos[l];
@@ -721,7 +802,6 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
     return CONST_OK;
 }
 
-
 // ------------------------------------------------------------------------------------------------
 // const_csf_build_noalloc: the same COO -> CSF pipeline with every temporary in one static device
 // array, for callers that must not allocate (see include/const_b200.h).
@@ -738,10 +818,11 @@ constexpr size_t kNaOffKeys1 = kNaOffKeys0 + kNaKeys;
 constexpr size_t kNaOffVals = kNaOffKeys1 + kNaKeys;                      // second payload buffer (the first is the caller's output)
 constexpr size_t kNaOffTileStatus = kNaOffVals + kNaKeys;
 constexpr size_t kNaOffHist = kNaOffTileStatus + sizeof(unsigned long long) * kNaTiles * kRsBins;
-constexpr size_t kNaOffBlockCounts = kNaOffHist + sizeof(uint32_t) * kMaxPasses * kRsBins;
-constexpr size_t kNaOffSmall = kNaOffBlockCounts + ((sizeof(uint32_t) * kCpLevels * kNaCpBlocks + 255) / 256) * 256;
-constexpr size_t kNaSmallBytes = 256;                                     // pass counters [8], level totals [4], status word
-constexpr size_t kNaBytes = kNaOffSmall + kNaSmallBytes;
+constexpr size_t kNaHistBytes = sizeof(uint32_t) * kMaxPasses * kRsBins;
+constexpr size_t kNaOffSmall = kNaOffHist + kNaHistBytes;                 // pass counters, level totals, status word
+constexpr size_t kNaSmallBytes = 256;
+constexpr size_t kNaOffBlockCounts = kNaOffSmall + kNaSmallBytes;
+constexpr size_t kNaBytes = kNaOffBlockCounts + ((sizeof(uint32_t) * kCpLevels * kNaCpBlocks + 255) / 256) * 256;
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress: it is not
 // a device address and must never be handed to a kernel or to cudaMemset as if it were one.
@@ -763,29 +844,6 @@ const_status_t noalloc_scratch(unsigned char **out) {
     return CONST_OK;
 }
 
-template <typename V>
-const_status_t noalloc_sort(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
-                            unsigned char *base, int32_t *status, cudaStream_t stream) {
-    uint32_t *hist = reinterpret_cast<uint32_t *>(base + kNaOffHist);
-    uint32_t *counters = reinterpret_cast<uint32_t *>(base + kNaOffSmall);
-    unsigned long long *tile_status = reinterpret_cast<unsigned long long *>(base + kNaOffTileStatus);
-    const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
-    int hist_blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
-    rs_histogram<<<hist_blocks, 256, 0, stream>>>(keys, n, passes, hist);
-    rs_scan_hist<<<passes, 256, 0, stream>>>(hist);
-    const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
-    CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-    for (int p = 0; p < passes; ++p) {
-        CB_CUDA(cudaMemsetAsync(tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
-        rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(keys, keys_alt, vals, vals_alt, n, 8 * p,
-                                                                     hist + p * kRsBins, tile_status, counters + p, status);
-        std::swap(keys, keys_alt);
-        std::swap(vals, vals_alt);
-    }
-    CB_CUDA(cudaGetLastError());
-    return CONST_OK;
-}
-
 }  // namespace
 
 const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
@@ -793,13 +851,8 @@ const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nn
                                       cudaStream_t stream, int32_t *const *pos_out, int32_t *const *crd_out,
                                       void *vals_out, int64_t *level_sizes) {
     if (nnz > kNoAllocMaxNnz) return CONST_ERR_WORKSPACE;
-    int bits[kMaxOrder] = {0, 0, 0, 0}, shift[kMaxOrder] = {0, 0, 0, 0};
-    int total_bits = 0;
-    for (int l = 0; l < order; ++l) { bits[l] = bits_for(dims[mode_order[l]]); total_bits += bits[l]; }
-    if (total_bits > 64) return CONST_ERR_UNSUPPORTED;
-    int acc = 0;
-    for (int l = order - 1; l >= 0; --l) { shift[l] = acc; acc += bits[l]; }
-    const int passes = (total_bits + 7) / 8;
+    KeyLayout kl;
+    if (!key_layout(order, dims, mode_order, kl)) return CONST_ERR_UNSUPPORTED;
 
     unsigned char *base = nullptr;
     const_status_t rc = noalloc_scratch(&base);
@@ -807,58 +860,45 @@ const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nn
     uint64_t *keys = reinterpret_cast<uint64_t *>(base + kNaOffKeys0);
     uint64_t *keys_alt = reinterpret_cast<uint64_t *>(base + kNaOffKeys1);
     uint32_t *block_counts = reinterpret_cast<uint32_t *>(base + kNaOffBlockCounts);
+    SortBufs sb{reinterpret_cast<uint32_t *>(base + kNaOffHist), reinterpret_cast<uint32_t *>(base + kNaOffSmall),
+                reinterpret_cast<unsigned long long *>(base + kNaOffTileStatus)};
     uint32_t *totals = reinterpret_cast<uint32_t *>(base + kNaOffSmall + 64);
     int32_t *status = reinterpret_cast<int32_t *>(base + kNaOffSmall + 128);
     // everything that must start at zero: digit histograms, pass counters, level totals, status word
-    CB_CUDA(cudaMemsetAsync(base + kNaOffHist, 0, sizeof(uint32_t) * kMaxPasses * kRsBins, stream));
-    CB_CUDA(cudaMemsetAsync(base + kNaOffSmall, 0, kNaSmallBytes, stream));
+    // (the tile states are cleared by the sort itself)
+    CB_CUDA(cudaMemsetAsync(base + kNaOffHist, 0, kNaHistBytes + kNaSmallBytes, stream));
 
     const size_t vsize = dtype == CONST_F32 ? 4 : 8;
     const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
     LevelShifts ls;
     ls.order = order;
-    for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = shift[l];
+    for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = kl.shift[l];
     if (nnz > 0) {
-        PackArgs pa;
-        pa.order = order;
-        for (int l = 0; l < kMaxOrder; ++l) {
-            pa.c[l] = l < order ? coords_dev[mode_order[l]] : nullptr;
-            pa.dim[l] = l < order ? dims[mode_order[l]] : 0;
-            pa.shift[l] = shift[l];
-        }
-        pack_keys<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(pa, nnz, keys, status);
+        PackArgs pa = pack_args(order, dims, mode_order, coords_dev, kl);
+        launch_pack_hist(pa, nnz, kl.passes, keys, sb.hist, status, stream);
         // the payload ping-pongs between the caller's output and the static buffer; start on the side
         // that makes the last pass land in the caller's output
-        void *va = vals_out, *vb = base + kNaOffVals;
-        void *first = (passes % 2 == 0) ? va : vb, *second = (passes % 2 == 0) ? vb : va;
+        void *first = (kl.passes % 2 == 0) ? vals_out : (void *)(base + kNaOffVals);
+        void *second = (kl.passes % 2 == 0) ? (void *)(base + kNaOffVals) : vals_out;
         CB_CUDA(cudaMemcpyAsync(first, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
-        if (dtype == CONST_F32) {
-            uint32_t *v = (uint32_t *)first, *w = (uint32_t *)second;
-            rc = noalloc_sort<uint32_t>(keys, keys_alt, v, w, nnz, passes, base, status, stream);
-        } else {
-            unsigned long long *v = (unsigned long long *)first, *w = (unsigned long long *)second;
-            rc = noalloc_sort<unsigned long long>(keys, keys_alt, v, w, nnz, passes, base, status, stream);
-        }
+        rc = sort_and_count(keys, keys_alt, first, second, nnz, kl.passes, dtype, sb, ls, block_counts, totals, status,
+                            stream);
         if (rc != CONST_OK) return rc;
-        csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status);
-        csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals);
     }
-    uint32_t h_totals[4] = {0, 0, 0, 0};
-    int32_t h_status = 0;
-    CB_CUDA(cudaMemcpyAsync(h_totals, totals, sizeof(h_totals), cudaMemcpyDeviceToHost, stream));
-    CB_CUDA(cudaMemcpyAsync(&h_status, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    uint32_t h_small[32] = {0};                   // totals at [0..4), status at [16]
+    CB_CUDA(cudaMemcpyAsync(h_small, totals, sizeof(uint32_t) * 17, cudaMemcpyDeviceToHost, stream));
     CB_CUDA(cudaStreamSynchronize(stream));
-    if (h_status != 0) return (const_status_t)h_status;
+    if (h_small[16] != 0) return (const_status_t)h_small[16];
     LevelSizes sz;
     sz.order = order;
     for (int l = 0; l < kMaxOrder; ++l) sz.n[l] = 0;
-    for (int l = 0; l < order - 1; ++l) sz.n[l] = h_totals[l];
+    for (int l = 0; l < order - 1; ++l) sz.n[l] = h_small[l];
     sz.n[order - 1] = nnz;
     CsfArrays arr;
     for (int l = 0; l < kMaxOrder; ++l) {
         arr.pos[l] = l < order ? pos_out[l] : nullptr;
         arr.crd[l] = l < order ? crd_out[l] : nullptr;
-        arr.bits[l] = bits[l];
+        arr.bits[l] = kl.bits[l];
     }
     if (nnz > 0) csf_scatter<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, arr);
     csf_finish<<<1, 32, 0, stream>>>(arr, sz);
