@@ -161,6 +161,8 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--impl", default="const")
     ap.add_argument("--oracle-nnz", type=int, default=0, help="nonzeros in the CPU-baseline sample (0 = auto)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
@@ -301,7 +303,7 @@ def main():
     h2d = sum(sum(c.numel() * c.element_size() for c in cs) + v.numel() * v.element_size() for cs, v in host.values())
     h2d += sum(a.numel() * a.element_size() for a in host_dense.values())
     d2h = out.numel() * out.element_size()
-    e2e_steps = max(2, min(args.steps, 5))
+    e2e_steps = 0 if args.kernels_only else max(2, min(args.steps, 5))
 
     def e2e_step():
         src = {n: ([c.cuda(non_blocking=True) for c in cs], v.cuda(non_blocking=True)) for n, (cs, v) in host.items()}
@@ -310,7 +312,8 @@ def main():
         out_host.copy_(out, non_blocking=True)
         free(hs)
 
-    e2e_step()
+    if e2e_steps:
+        e2e_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -318,7 +321,7 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps if e2e_steps else float("nan")
     if dist is not None:
         t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -373,7 +376,7 @@ def main():
 
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ----
     auto = {1: 20_000, 2: 40_000_000, 3: 8_000_000, 4: 100_000_000, 5: 400_000}[args.config]
-    cpu_baseline, _ = time_oracle(w, args.oracle_nnz or auto)
+    cpu_baseline = None if args.kernels_only else time_oracle(w, args.oracle_nnz or auto)[0]
 
     line = {
         "metric": "useful GFLOP/s", "value": total_flops * world / world / (ms_per_step * 1e-3) / 1e9,

@@ -735,8 +735,8 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
         auto body = [&]() -> const_status_t {
             CB_CUDA(tmp.alloc((void **)&keys, sizeof(uint64_t) * nnz));
             CB_CUDA(tmp.alloc((void **)&keys_alt, sizeof(uint64_t) * nnz));
-            CB_CUDA(tmp.alloc(&vals, vsize * nnz));
-            CB_CUDA(tmp.alloc(&vals_alt, vsize * nnz));
+            CB_CUDA(tmp.alloc(&vals, vsize * (nnz + 4)));
+            CB_CUDA(tmp.alloc(&vals_alt, vsize * (nnz + 4)));
             CB_CUDA(tmp.alloc((void **)&small, kSmallBytes));
             CB_CUDA(tmp.alloc((void **)&sb.tile_status, sizeof(unsigned long long) * std::max<int64_t>(ntiles, 1) * kRsBins));
             CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * kCpLevels * std::max<int64_t>(cp_blocks, 1)));
@@ -768,7 +768,7 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             for (int l = 0; l < order; ++l) {
                 const int64_t parents = l == 0 ? 1 : csf->n[l - 1];
                 CB_CUDA(pool_alloc((void **)&csf->pos[l], sizeof(int32_t) * (parents + 1), stream));
-                CB_CUDA(pool_alloc((void **)&csf->crd[l], sizeof(int32_t) * std::max<int64_t>(csf->n[l], 1), stream));
+                CB_CUDA(pool_alloc((void **)&csf->crd[l], sizeof(int32_t) * (csf->n[l] + 4), stream));
                 arr.pos[l] = csf->pos[l];
                 arr.crd[l] = csf->crd[l];
             }
