@@ -103,15 +103,16 @@ __global__ void __launch_bounds__(256) rs_scan_hist(uint32_t *hist) {
 }
 
 template <typename V>
-__global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__restrict__ kin, uint64_t *__restrict__ kout,
-                                                         const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
-                                                         int shift, const uint32_t *__restrict__ digit_base,
-                                                         unsigned long long *status, uint32_t *counter,
-                                                         int32_t *err, unsigned epoch) {
+__global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__restrict__ kin, uint64_t *__restrict__ kout,
+                                                            const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
+                                                            int shift, const uint32_t *__restrict__ digit_base,
+                                                            unsigned long long *status, uint32_t *counter,
+                                                            int32_t *err, unsigned epoch) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t *keybuf = reinterpret_cast<uint64_t *>(smem_raw);
     V *valbuf = reinterpret_cast<V *>(smem_raw + kRsTile * sizeof(uint64_t));
     __shared__ uint32_t warp_hist[kRsWarps][kRsBins];
+    __shared__ uint32_t tile_hist[kRsBins];
     __shared__ uint32_t digit_excl[kRsBins];
     __shared__ long long s_gbase[kRsBins];
     __shared__ uint32_t warp_tot[kRsWarps];
@@ -121,47 +122,62 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) { s_tile = atomicAdd(counter, 1u); s_abort = 0; }
     for (int x = threadIdx.x; x < kRsWarps * kRsBins; x += kRsThreads) (&warp_hist[0][0])[x] = 0;
+    tile_hist[threadIdx.x] = 0;
     __syncthreads();
     const int64_t tile = s_tile;
     const int64_t tile_base = tile * kRsTile;
     if (tile_base >= n) return;                       // never happens: the grid has exactly ceil(n / tile) blocks
 
     uint64_t key[kRsItems];
-    V val[kRsItems];
 #pragma unroll
     for (int i = 0; i < kRsItems; ++i) {
         int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
-        bool in = idx < n;
-        key[i] = in ? kin[idx] : ~0ull;               // padding sorts after every real key of the tile
-        val[i] = in ? vin[idx] : V(0);
+        key[i] = idx < n ? kin[idx] : ~0ull;          // padding sorts after every real key of the tile
     }
 
-    // rank inside the warp: keys with equal digits keep their order (item, lane)
+    // Digit counts of the tile first, so that later tiles can see them as early as possible:
+    // the time from taking a tile to publishing its counts decides how long others wait.
+#pragma unroll
+    for (int i = 0; i < kRsItems; ++i) atomicAdd(&tile_hist[(unsigned)(key[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    const int d = threadIdx.x;                        // thread d owns digit d from here on
+    const uint32_t count = tile_hist[d];
+    volatile unsigned long long *st = status;
+    // A status word counts only if it carries this pass's number, so the array is cleared once per
+    // sort, not once per pass.
+    const unsigned long long tag = (unsigned long long)epoch << 32;
+    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | tag | (unsigned long long)count;
+
+    // Rank inside the warp: keys with equal digits keep their order (item, lane).  peers = lanes
+    // holding the same digit, from one ballot per digit bit (the match instruction costs one round
+    // per distinct value in the warp, which for random digits is far slower).
     int rank[kRsItems];
 #pragma unroll
     for (int i = 0; i < kRsItems; ++i) {
-        unsigned d = (unsigned)(key[i] >> shift) & 255u;
-        unsigned peers = __match_any_sync(0xffffffffu, d);
-        int leader = __ffs(peers) - 1;
-        uint32_t old = 0;
-        if (lane == leader) {
-            old = warp_hist[warp][d];
-            warp_hist[warp][d] = old + __popc(peers);
+        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
+        unsigned peers = 0xffffffffu;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const unsigned bit = (dg >> b) & 1u;
+            peers &= __ballot_sync(0xffffffffu, bit) ^ (bit - 1u);      // lanes whose bit b equals mine
         }
+        const int leader = __ffs(peers) - 1;
+        uint32_t old = 0;
+        if (lane == leader) old = atomicAdd(&warp_hist[warp][dg], (uint32_t)__popc(peers));
         old = __shfl_sync(0xffffffffu, old, leader);
         rank[i] = (int)old + __popc(peers & ((1u << lane) - 1u));
-        __syncwarp();
     }
     __syncthreads();
 
-    // thread d owns digit d: offsets of each warp's run, tile total, digit scan inside the tile
-    const int d = threadIdx.x;
-    uint32_t count = 0;
+    // offsets of each warp's run inside the digit, digit scan inside the tile
+    {
+        uint32_t run = 0;
 #pragma unroll
-    for (int w = 0; w < kRsWarps; ++w) {
-        uint32_t c = warp_hist[w][d];
-        warp_hist[w][d] = count;
-        count += c;
+        for (int w = 0; w < kRsWarps; ++w) {
+            uint32_t c = warp_hist[w][d];
+            warp_hist[w][d] = run;
+            run += c;
+        }
     }
     uint32_t incl = count;
 #pragma unroll
@@ -176,28 +192,34 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
     const uint32_t excl_in_tile = wbase + incl - count;
 
     // chained scan over tiles (decoupled look-back); every wait is bounded
-    volatile unsigned long long *st = status;
-    // A status word counts only if it carries this pass's number, so the array is cleared once per
-    // sort, not once per pass.
-    const unsigned long long tag = (unsigned long long)epoch << 32;
-    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | tag | (unsigned long long)count;
     unsigned long long before = 0;
     if (tile > 0) {
-        bool ok = true;
+        // The states of kLook predecessors are requested together, so a walk over tiles that have
+        // only published their own counts costs one memory round trip per kLook tiles.
+        constexpr int kLook = 8;
+        bool ok = true, done = false;
         int64_t t = tile - 1;
-        for (;;) {
-            unsigned long long s = 0;
-            int spins = 0;
-            for (;;) {
-                s = st[t * kRsBins + d];
-                if ((s >> 62) && ((s >> 32) & 0xffu) == epoch) break;
-                if (++spins > kSpinLimit) { ok = false; break; }
-                if (spins > 64) __nanosleep(100);
+        while (ok && !done) {
+            unsigned long long s[kLook];
+#pragma unroll
+            for (int b = 0; b < kLook; ++b) s[b] = t - b >= 0 ? st[(t - b) * kRsBins + d] : 0ull;
+#pragma unroll
+            for (int b = 0; b < kLook; ++b) {
+                if (ok && !done && t - b >= 0) {
+                    unsigned long long v = s[b];
+                    int spins = 0;
+                    while (!((v >> 62) && ((v >> 32) & 0xffu) == epoch)) {
+                        if (++spins > kSpinLimit) { ok = false; break; }
+                        if (spins > 64) __nanosleep(100);
+                        v = st[(t - b) * kRsBins + d];
+                    }
+                    if (ok) {
+                        before += v & kValMask;
+                        if ((v >> 62) == 2ull || t - b == 0) done = true;
+                    }
+                }
             }
-            if (!ok) break;
-            before += s & kValMask;
-            if ((s >> 62) == 2ull || t == 0) break;
-            --t;
+            t -= kLook;
         }
         if (ok) {
             st[tile * kRsBins + d] = kFlagInc | tag | (before + count);
@@ -211,13 +233,16 @@ __global__ void __launch_bounds__(kRsThreads) rs_onesweep(const uint64_t *__rest
     __syncthreads();
     if (s_abort) return;
 
-    // reorder in shared memory, then store runs of consecutive addresses
+    // reorder in shared memory (the payload is fetched only now: it is not needed for ranking),
+    // then store runs of consecutive addresses
 #pragma unroll
     for (int i = 0; i < kRsItems; ++i) {
-        unsigned dg = (unsigned)(key[i] >> shift) & 255u;
-        int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
+        const int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
+        const V val = idx < n ? vin[idx] : V(0);
+        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
+        const int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
         keybuf[p] = key[i];
-        valbuf[p] = val[i];
+        valbuf[p] = val;
     }
     __syncthreads();
     const int64_t left = n - tile_base;
