@@ -112,6 +112,19 @@ def time_oracle(w, target_nnz):
             "sample": f"{len(rows)} seeded output rows holding {sub.nnz} nonzeros, {dt:.2f} s"}, dt
 
 
+def aggregate_over_ranks(ms_per_step, work, dist=None, device="cpu"):
+    """Whole-job figures for independent replicas (one per rank, no data-path collective):
+    the step time is the maximum over ranks, the work done is the sum over ranks."""
+    if dist is None:
+        return float(ms_per_step), float(work)
+    import torch
+    t = torch.tensor([float(ms_per_step)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    f = torch.tensor([float(work)], device=device, dtype=torch.float64)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(f.item())
+
+
 # ------------------------------------------------------------------------------------------------
 # clocks sampler
 # ------------------------------------------------------------------------------------------------
@@ -126,7 +139,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
@@ -155,7 +168,7 @@ class ClockSampler:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--scale", type=float, default=1.0)
@@ -289,15 +302,7 @@ def main():
     cb.const_profile_enable(False)
     clocks = sampler.stop()
     ms_per_step = total_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_per_step], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
-        f = torch.tensor([float(flops)], device="cuda", dtype=torch.float64)
-        dist.all_reduce(f, op=dist.ReduceOp.SUM)
-        total_flops = float(f.item())
-    else:
-        total_flops = float(flops)
+    ms_per_step, total_flops = aggregate_over_ranks(ms_per_step, flops, dist, "cuda")
 
     # ---- end to end: host buffers in, result out ----
     h2d = sum(sum(c.numel() * c.element_size() for c in cs) + v.numel() * v.element_size() for cs, v in host.values())
@@ -322,10 +327,7 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps if e2e_steps else float("nan")
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms, _ = aggregate_over_ranks(e2e_ms, flops, dist, "cuda")
 
     if rank != 0:
         if dist is not None:
@@ -379,7 +381,7 @@ def main():
     cpu_baseline = None if args.kernels_only else time_oracle(w, args.oracle_nnz or auto)[0]
 
     line = {
-        "metric": "useful GFLOP/s", "value": total_flops * world / world / (ms_per_step * 1e-3) / 1e9,
+        "metric": "useful GFLOP/s", "value": total_flops / (ms_per_step * 1e-3) / 1e9,
         "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if dtype == cb.F32 else "f64", "data": "synthetic",
