@@ -160,7 +160,7 @@ const_status_t const_csf_bin_counts(const const_csf_t *csf, int64_t *n_light, in
  *           8, 16 or 32 (order-4 TTMc: 8).  The loops above each contracted level must be fused, so
  *           intermediates reduce to order 1 (order 2 for the middle one of order-4 TTMc).  CONST_F32.
  *   network T[i,k,l] = U[i,j,k] * V[j,l]; Z[i,m] = T[i,k,l] * W[k,l,m] with V dense, U in CSF with
- *           levels (i,k,j) and W in CSF with levels (m,l,k), loop orders i,k,j,l and i,m,l,k: both
+ *           levels (i,k,j) and W in CSF with levels (l,m,k), loop orders i,k,j,l and i,l,m,k: both
  *           contractions then gather along a fibre; fused over i only (T reduced to order 2).  CONST_F64.
  */
 const_status_t const_plan_create(const char *expression, const char *const *tree, int n_contractions,

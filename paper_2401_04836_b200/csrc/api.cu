@@ -214,10 +214,10 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
             if (!w || !w->csf || w->dense_dev) return CONST_ERR_INVALID_ARG;
             const const_csf *W = as_csf(w->csf);
             if (!csf_matches(W, d, d.sparse2_name, d.dtype)) return CONST_ERR_INVALID_ARG;
-            // level extents of U (i,k,j) and W (m,l,k)
+            // level extents of U (i,k,j) and W (l,m,k)
             const int64_t n_i = X->dims[X->mode_order[0]], n_k = X->dims[X->mode_order[1]],
                           n_j = X->dims[X->mode_order[2]];
-            const int64_t n_m = W->dims[W->mode_order[0]], n_l = W->dims[W->mode_order[1]];
+            const int64_t n_l = W->dims[W->mode_order[0]], n_m = W->dims[W->mode_order[1]];
             return run_network(X, (const double *)dense[0], W, (double *)out_dev, n_i, n_j, n_k, n_l, n_m,
                                p->status_dev, stream);
         }

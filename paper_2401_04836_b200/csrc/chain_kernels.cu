@@ -60,7 +60,7 @@ struct Shape {
     // phase 1
     static constexpr int LPR1 = R3 / 4;                 // lanes per factor row
     static constexpr int G1 = 32 / LPR1;                // lane groups per warp
-    static constexpr int WINDOW = R3 >= 32 ? 32 : 64;   // fibres parked per warp
+    static constexpr int WINDOW = R3 >= 32 ? 64 : 128;  // fibres parked per warp
     // phase 2: register block of RW rows x 4 columns per lane
     static constexpr int RW = HADAMARD ? 1 : 8;
     static constexpr int LPF = HADAMARD ? R3 / 4 : (R2 / 8) * (R3 / 4);   // lanes that cover one fibre
@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 chain3_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ light_list, Csf3 x,
               const float *__restrict__ F1, const float *__restrict__ F2, float *__restrict__ out) {
     using S = Shape<R2, R3, HADAMARD>;
-    __shared__ __align__(16) float Ts_all[kWarpsPerBlock][S::WINDOW * R3];
+    extern __shared__ __align__(16) float Ts_all[];          // [warp][WINDOW * R3] parked rows
     __shared__ int32_t Js_all[kWarpsPerBlock][S::WINDOW];
     __shared__ int32_t Ps_all[kWarpsPerBlock][S::WINDOW + 1];
     __shared__ __align__(16) float Hs_all[kWarpsPerBlock][S::G1 * R3];
@@ -268,7 +268,7 @@ chain3_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ li
     float acc[S::NACC];
 #pragma unroll
     for (int a = 0; a < S::NACC; ++a) acc[a] = 0.f;
-    float *Ts = Ts_all[warp];
+    float *Ts = Ts_all + warp * (S::WINDOW * R3);
     int32_t *Js = Js_all[warp];
     for (int32_t s0 = fa; s0 < fb; s0 += S::WINDOW) {
         const int cnt = fb - s0 < S::WINDOW ? fb - s0 : S::WINDOW;
@@ -317,8 +317,17 @@ const_status_t launch_chain3(const const_csf *X, const float *F1, const float *F
     CB_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * TILE * n_rows, stream));       // "R[*] = 0" precedes the nest
     if (X->n_items == 0) return CONST_OK;
     Csf3 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], static_cast<const float *>(X->vals)};
+    using S = Shape<R2, R3, HADAMARD>;
+    constexpr size_t dyn = sizeof(float) * kWarpsPerBlock * S::WINDOW * R3;
+    static bool attr_set[64] = {false};                     // per template instance and device
+    int dev = 0;
+    CB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        CB_CUDA(cudaFuncSetAttribute(chain3_kernel<R2, R3, HADAMARD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
     CB_LAUNCH("chain3_kernel", stream,
-              chain3_kernel<R2, R3, HADAMARD><<<(unsigned)X->n_items, kWarpsPerBlock * 32, 0, stream>>>(
+              chain3_kernel<R2, R3, HADAMARD><<<(unsigned)X->n_items, kWarpsPerBlock * 32, dyn, stream>>>(
                   X->items, X->light_list, x, F1, F2, out));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;

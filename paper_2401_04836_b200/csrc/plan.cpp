@@ -342,12 +342,12 @@ const_status_t match_plan(PlanDesc &p) {
         if (U->idx.size() != 3 || W->idx.size() != 3 || V->idx.size() != 2 || T->idx.size() != 3 ||
             p.result.idx.size() != 2)
             return no("network family needs order-3 sparse tensors and a dense matrix");
-        // gather-form schedule: U stored (i,k,j), W stored (m,l,k)
+        // gather-form schedule: U stored (i,k,j), W stored (l,m,k)
         const std::vector<int> &mu = p.mode_orders[U->name], &mw = p.mode_orders[W->name];
         char i = U->idx[mu[0]], k = U->idx[mu[1]], j = U->idx[mu[2]];
-        char mm = W->idx[mw[0]], l = W->idx[mw[1]], wk = W->idx[mw[2]];
-        if (wk != k) return no("W's leaf level must be the index it shares with U (U stored i,k,j; W stored m,l,k)");
-        if (V->idx[0] != j || V->idx[1] != l) return no("V must be indexed [U's leaf index, W's middle index]");
+        char l = W->idx[mw[0]], mm = W->idx[mw[1]], wk = W->idx[mw[2]];
+        if (wk != k) return no("W's leaf level must be the index it shares with U (U stored i,k,j; W stored l,m,k)");
+        if (V->idx[0] != j || V->idx[1] != l) return no("V must be indexed [U's leaf index, W's root index]");
         std::string t = T->idx;
         std::sort(t.begin(), t.end());
         std::string want{i, k, l};

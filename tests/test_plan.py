@@ -133,8 +133,9 @@ def test_network_schedule_variants():
     # scatter-form schedule (U stored i,j,k; W stored k,l,m) is legal but has no kernel here
     assert mk(mode_orders={"U": (0, 1, 2), "W": (0, 1, 2)}, loop_orders=["ijkl", "iklm"]) == 2
     # not fused over i: T stays order 3
-    assert mk(loop_orders=["ikjl", "milk"]) == 2               # legal, but T keeps all three modes
-    assert mk(loop_orders=["ikjl", "ilmk"]) == 3               # W stored (m,l,k): l may not precede m
+    assert mk(loop_orders=["ikjl", "lmik"]) == 2               # legal, but T keeps all three modes
+    assert mk(loop_orders=["ikjl", "imlk"]) == 3               # W stored (l,m,k): m may not precede l
+    assert mk(mode_orders={"U": (0, 2, 1), "W": (2, 1, 0)}, loop_orders=["ikjl", "imlk"]) == 2   # W as (m,l,k)
     assert mk(dtype=cb.F32) == 2
 
 

@@ -334,7 +334,7 @@ def network_workload(n=1024, n_k=128, band=32, keep=0.25, *, seed=0, config_id=5
         sparse={"U": U, "W": W}, dense={"V": V},
         expression="Z[i,m] = U[i,j,k] * V[j,l] * W[k,l,m]",
         tree=["T[i,k,l] = U[i,j,k] * V[j,l]", "Z[i,m] = T[i,k,l] * W[k,l,m]"],
-        mode_orders={"U": (0, 2, 1), "W": (2, 1, 0)}, loop_orders=["ikjl", "imlk"],
+        mode_orders={"U": (0, 2, 1), "W": (1, 2, 0)}, loop_orders=["ikjl", "ilmk"],
         out_shape=(n, n))
 
 
