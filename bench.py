@@ -32,6 +32,11 @@ if ROOT not in sys.path:
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 
+# DRAM bytes per nonzero and launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of
+# config 2 at scale 0.3 summarised under profiles/; both kernels stream their inputs once, so the traffic
+# of a full-size launch is this figure times its nonzero count.  Only valid for that workload family.
+NCU_TRAFFIC_BYTES_PER_NNZ = {("ttmc3", "rs_onesweep"): 526.0e6 / 23.1e6, ("ttmc3", "chain3_kernel"): 236.6e6 / 23.1e6}
+
 
 def measured_peaks():
     try:
@@ -344,7 +349,17 @@ def main():
     fused_names = {"chain3_kernel", "ttmc4_kernel", "network_kernel"}
     vbytes = w.dtype.itemsize
 
+    def traffic_of(name):
+        per = NCU_TRAFFIC_BYTES_PER_NNZ.get((w.family, name))
+        return None if per is None else per * nnz_total / len(w.sparse)
+
     def roofline_of(name):
+        r = _roofline_of(name)
+        if r is not None:
+            r["traffic"] = traffic_of(name)
+        return r
+
+    def _roofline_of(name):
         n, ms = prof[name]
         per_launch_ms = ms / n
         if name in fused_names:
