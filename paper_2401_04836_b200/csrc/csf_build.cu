@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
                     int spins = 0;
                     while (!((v >> 62) && ((v >> 32) & 0xffu) == epoch)) {
                         if (++spins > kSpinLimit) { ok = false; break; }
-                        if (spins > 64) __nanosleep(100);
+                        __nanosleep(spins < 8 ? 200 : 1000);   // back off at once: polling warps must not crowd the issue slots
                         v = st[(t - b) * kRsBins + d];
                     }
                     if (ok) {
