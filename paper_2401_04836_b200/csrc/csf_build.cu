@@ -190,6 +190,21 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     uint32_t wbase = 0;
     for (int w = 0; w < warp; ++w) wbase += warp_tot[w];
     const uint32_t excl_in_tile = wbase + incl - count;
+    digit_excl[d] = excl_in_tile;
+    __syncthreads();
+
+    // Reorder in shared memory first (the payload is fetched only now: it is not needed for ranking).
+    // This needs tile-local offsets only, so it runs before the look-back: by the time the global
+    // prefix is needed, most predecessors have published theirs and little time is spent polling.
+#pragma unroll
+    for (int i = 0; i < kRsItems; ++i) {
+        const int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
+        const V val = idx < n ? vin[idx] : V(0);
+        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
+        const int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
+        keybuf[p] = key[i];
+        valbuf[p] = val;
+    }
 
     // chained scan over tiles (decoupled look-back); every wait is bounded
     unsigned long long before = 0;
@@ -228,23 +243,11 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
             s_abort = 1;
         }
     }
-    digit_excl[d] = excl_in_tile;
     s_gbase[d] = (long long)digit_base[d] + (long long)before - (long long)excl_in_tile;
     __syncthreads();
     if (s_abort) return;
 
-    // reorder in shared memory (the payload is fetched only now: it is not needed for ranking),
-    // then store runs of consecutive addresses
-#pragma unroll
-    for (int i = 0; i < kRsItems; ++i) {
-        const int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
-        const V val = idx < n ? vin[idx] : V(0);
-        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
-        const int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
-        keybuf[p] = key[i];
-        valbuf[p] = val;
-    }
-    __syncthreads();
+    // store runs of consecutive addresses
     const int64_t left = n - tile_base;
     const int nvalid = left < kRsTile ? (int)left : kRsTile;
 #pragma unroll
