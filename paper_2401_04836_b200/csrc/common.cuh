@@ -26,7 +26,7 @@ struct WorkItem {
 };
 
 constexpr int kItemLight = 0, kItemBlock = 1, kItemChunk = 2;
-constexpr int kWarpsPerBlock = 8;             // fused kernels run 256-thread blocks
+constexpr int kWarpsPerBlock = 2;             // fused kernels run 64-thread blocks (small blocks keep warp slots busy)
 
 }  // namespace cb
 
