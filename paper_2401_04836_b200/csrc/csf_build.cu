@@ -743,9 +743,9 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
     csf->stream = stream;
     cudaGetDevice(&csf->device);
     for (int l = 0; l < order; ++l) { csf->dims[l] = dims[l]; csf->mode_order[l] = mode_order[l]; }
-    csf->light_max = 1024;
-    csf->heavy_max = 12288;
-    csf->chunk = 6144;
+    csf->light_max = 2048;
+    csf->heavy_max = 16384;
+    csf->chunk = 8192;
 
     const size_t vsize = dtype == CONST_F32 ? 4 : 8;
     const_status_t rc = CONST_OK;
