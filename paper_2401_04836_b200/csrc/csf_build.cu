@@ -35,17 +35,23 @@ enum DevErr : int32_t { kErrNone = 0 };
 
 __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicCAS(status, 0, code); }
 
-constexpr int kRsBins = 256;
+constexpr int kRsMaxBits = 9;                     // widest digit of a radix pass
+constexpr int kRsMaxBins = 1 << kRsMaxBits;
 constexpr int kMaxPasses = 8;
 
+// Digits of the radix passes.  A pass sorts on `bits[p]` key bits starting at `shift[p]`; the widths
+// are 8 or 9 bits (the width the pass kernel is instantiated for), chosen so that the key is covered
+// in as few passes as possible.
+struct DigitPlan { int shift[kMaxPasses]; int bits[kMaxPasses]; int passes; };
+
 // Pack the permuted coordinates of every nonzero into its 64-bit sort key (range-checked) and, in the
-// same read, count the 8-bit digits of every radix pass.  Per-block counts live in shared memory and
-// are flushed once; the grid is sized to a few blocks per SM so the flush stays small.
+// same read, count the digits of every radix pass.  Per-block counts live in shared memory and are
+// flushed once; the grid is sized to a few blocks per SM so the flush stays small.
 template <int ORDER>
-__global__ void __launch_bounds__(256) pack_hist(PackArgs a, int64_t nnz, int passes, uint64_t *__restrict__ keys,
+__global__ void __launch_bounds__(256) pack_hist(PackArgs a, int64_t nnz, DigitPlan dp, uint64_t *__restrict__ keys,
                                                  uint32_t *__restrict__ hist, int32_t *status) {
-    __shared__ uint32_t sh[kMaxPasses * kRsBins];
-    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x) sh[x] = 0;
+    extern __shared__ uint32_t sh[];                 // [passes][kRsMaxBins]
+    for (int x = threadIdx.x; x < dp.passes * kRsMaxBins; x += blockDim.x) sh[x] = 0;
     __syncthreads();
     bool bad = false;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -58,21 +64,23 @@ __global__ void __launch_bounds__(256) pack_hist(PackArgs a, int64_t nnz, int pa
             key |= (uint64_t)c << a.shift[l];
         }
         keys[e] = key;
-        for (int p = 0; p < passes; ++p) atomicAdd(&sh[p * kRsBins + ((unsigned)(key >> (8 * p)) & 255u)], 1u);
+        for (int p = 0; p < dp.passes; ++p)
+            atomicAdd(&sh[p * kRsMaxBins + ((unsigned)(key >> dp.shift[p]) & ((1u << dp.bits[p]) - 1u))], 1u);
     }
     if (bad) report(status, CONST_ERR_COORD_RANGE);
     __syncthreads();
-    for (int x = threadIdx.x; x < passes * kRsBins; x += blockDim.x)
+    for (int x = threadIdx.x; x < dp.passes * kRsMaxBins; x += blockDim.x)
         if (sh[x]) atomicAdd(&hist[x], sh[x]);
 }
 
-inline void launch_pack_hist(const PackArgs &pa, int64_t nnz, int passes, uint64_t *keys, uint32_t *hist,
+inline void launch_pack_hist(const PackArgs &pa, int64_t nnz, const DigitPlan &dp, uint64_t *keys, uint32_t *hist,
                              int32_t *status, cudaStream_t stream) {
     const int blocks = (int)std::min<int64_t>((nnz + 255) / 256, 148 * 8);
+    const size_t sm = sizeof(uint32_t) * kRsMaxBins * std::max(dp.passes, 1);
     switch (pa.order) {
-        case 2: pack_hist<2><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
-        case 3: pack_hist<3><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
-        default: pack_hist<4><<<blocks, 256, 0, stream>>>(pa, nnz, passes, keys, hist, status); break;
+        case 2: pack_hist<2><<<blocks, 256, sm, stream>>>(pa, nnz, dp, keys, hist, status); break;
+        case 3: pack_hist<3><<<blocks, 256, sm, stream>>>(pa, nnz, dp, keys, hist, status); break;
+        default: pack_hist<4><<<blocks, 256, sm, stream>>>(pa, nnz, dp, keys, hist, status); break;
     }
 }
 
@@ -83,84 +91,101 @@ constexpr int kRsThreads = 256;
 constexpr int kRsItems = 16;
 constexpr int kRsTile = kRsThreads * kRsItems;     // 4096 keys per tile
 constexpr int kRsWarps = kRsThreads / 32;
-constexpr uint64_t kFlagAgg = 1ull << 62;          // tile published its own digit counts
-constexpr uint64_t kFlagInc = 2ull << 62;          // tile published counts summed over all earlier tiles too
-constexpr uint64_t kValMask = (1ull << 32) - 1;       // low 32 bits: count; bits 32..39: pass number + 1
 constexpr int kSpinLimit = 1 << 21;
+// A tile's state for one digit is one 64-bit word: the count in the low half; in the high half
+// (pass number << 2) | flag, flag 1 = the tile's own count, flag 2 = the count summed over this and
+// every earlier tile.  A word counts only if it carries the current pass number, so the array is
+// cleared once per sort, not once per pass.
+constexpr unsigned kFlagOwn = 1u, kFlagPrefix = 2u;
 
-// Exclusive scan of each pass's 256-bin histogram: one block per pass.
+__device__ __forceinline__ unsigned long long status_word(unsigned epoch, unsigned flag, uint32_t count) {
+    return ((unsigned long long)((epoch << 2) | flag) << 32) | count;
+}
+
+// Exclusive scan of each pass's digit histogram: one block per pass.
 __global__ void __launch_bounds__(256) rs_scan_hist(uint32_t *hist) {
-    __shared__ uint32_t sh[kRsBins];
-    uint32_t *h = hist + blockIdx.x * kRsBins;
-    sh[threadIdx.x] = h[threadIdx.x];
+    __shared__ uint32_t sh[kRsMaxBins];
+    uint32_t *h = hist + blockIdx.x * kRsMaxBins;
+    for (int x = threadIdx.x; x < kRsMaxBins; x += blockDim.x) sh[x] = h[x];
     __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t run = 0;
-        for (int d = 0; d < kRsBins; ++d) { uint32_t c = sh[d]; sh[d] = run; run += c; }
+        for (int d = 0; d < kRsMaxBins; ++d) { uint32_t c = sh[d]; sh[d] = run; run += c; }
     }
     __syncthreads();
-    h[threadIdx.x] = sh[threadIdx.x];
+    for (int x = threadIdx.x; x < kRsMaxBins; x += blockDim.x) h[x] = sh[x];
 }
 
-template <typename V>
+// One radix pass over BITS key bits.  Thread t owns digits t, t + 256, ... (DPT of them).
+template <typename V, int BITS>
 __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__restrict__ kin, uint64_t *__restrict__ kout,
                                                             const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
                                                             int shift, const uint32_t *__restrict__ digit_base,
                                                             unsigned long long *status, uint32_t *counter,
                                                             int32_t *err, unsigned epoch) {
+    constexpr int kBins = 1 << BITS;
+    constexpr unsigned kDigitMask = kBins - 1;
+    constexpr int DPT = kBins / kRsThreads;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t *keybuf = reinterpret_cast<uint64_t *>(smem_raw);
     V *valbuf = reinterpret_cast<V *>(smem_raw + kRsTile * sizeof(uint64_t));
-    __shared__ uint32_t warp_hist[kRsWarps][kRsBins];
-    __shared__ uint32_t tile_hist[kRsBins];
-    __shared__ uint32_t digit_excl[kRsBins];
-    __shared__ long long s_gbase[kRsBins];
-    __shared__ uint32_t warp_tot[kRsWarps];
+    __shared__ uint32_t warp_hist[kRsWarps][kBins];
+    __shared__ uint32_t tile_hist[kBins];
+    __shared__ uint32_t digit_excl[kBins];
+    __shared__ uint32_t s_gbase[kBins];
+    __shared__ uint32_t warp_tot[DPT][kRsWarps];
     __shared__ uint32_t s_tile;
     __shared__ int s_abort;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) { s_tile = atomicAdd(counter, 1u); s_abort = 0; }
-    for (int x = threadIdx.x; x < kRsWarps * kRsBins; x += kRsThreads) (&warp_hist[0][0])[x] = 0;
-    tile_hist[threadIdx.x] = 0;
+    for (int x = threadIdx.x; x < kRsWarps * kBins; x += kRsThreads) (&warp_hist[0][0])[x] = 0;
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) tile_hist[q * kRsThreads + threadIdx.x] = 0;
     __syncthreads();
-    const int64_t tile = s_tile;
-    const int64_t tile_base = tile * kRsTile;
+    const uint32_t tile = s_tile;
+    const int64_t tile_base = (int64_t)tile * kRsTile;
     if (tile_base >= n) return;                       // never happens: the grid has exactly ceil(n / tile) blocks
+    const int64_t left = n - tile_base;
+    const int nvalid = left < kRsTile ? (int)left : kRsTile;
 
+    // this thread's slots of the tile: local indices mine + 32 i
+    const int mine = warp * (32 * kRsItems) + lane;
+    const uint64_t *ktile = kin + tile_base + mine;
     uint64_t key[kRsItems];
 #pragma unroll
-    for (int i = 0; i < kRsItems; ++i) {
-        int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
-        key[i] = idx < n ? kin[idx] : ~0ull;          // padding sorts after every real key of the tile
-    }
+    for (int i = 0; i < kRsItems; ++i)
+        key[i] = mine + i * 32 < nvalid ? ktile[i * 32] : ~0ull;   // padding sorts after every real key of the tile
 
     // Digit counts of the tile first, so that later tiles can see them as early as possible:
     // the time from taking a tile to publishing its counts decides how long others wait.
 #pragma unroll
-    for (int i = 0; i < kRsItems; ++i) atomicAdd(&tile_hist[(unsigned)(key[i] >> shift) & 255u], 1u);
+    for (int i = 0; i < kRsItems; ++i) atomicAdd(&tile_hist[(unsigned)(key[i] >> shift) & kDigitMask], 1u);
     __syncthreads();
-    const int d = threadIdx.x;                        // thread d owns digit d from here on
-    const uint32_t count = tile_hist[d];
     volatile unsigned long long *st = status;
-    // A status word counts only if it carries this pass's number, so the array is cleared once per
-    // sort, not once per pass.
-    const unsigned long long tag = (unsigned long long)epoch << 32;
-    st[tile * kRsBins + d] = (tile == 0 ? kFlagInc : kFlagAgg) | tag | (unsigned long long)count;
+    uint32_t count[DPT];
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = q * kRsThreads + threadIdx.x;
+        count[q] = tile_hist[d];
+        st[(size_t)tile * kBins + d] = status_word(epoch, tile == 0 ? kFlagPrefix : kFlagOwn, count[q]);
+    }
 
-    // Rank inside the warp: keys with equal digits keep their order (item, lane).  peers = lanes
-    // holding the same digit, from one ballot per digit bit (the match instruction costs one round
-    // per distinct value in the warp, which for random digits is far slower).
+    // Rank inside the warp: keys with equal digits keep their order (item, lane).  The lanes holding
+    // another digit are collected from one ballot per digit bit (the match instruction costs one
+    // round per distinct value in the warp, which for random digits is far slower).
     int rank[kRsItems];
 #pragma unroll
     for (int i = 0; i < kRsItems; ++i) {
-        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
-        unsigned peers = 0xffffffffu;
+        const unsigned dg = (unsigned)(key[i] >> shift) & kDigitMask;
+        unsigned other = 0;
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            const unsigned bit = (dg >> b) & 1u;
-            peers &= __ballot_sync(0xffffffffu, bit) ^ (bit - 1u);      // lanes whose bit b equals mine
+        for (int b = 0; b < BITS; ++b) {
+            const bool bit = (dg >> b) & 1u;
+            const unsigned m = __ballot_sync(0xffffffffu, bit);
+            other |= bit ? ~m : m;                                     // lanes whose bit b differs from mine
         }
+        const unsigned peers = ~other;
         const int leader = __ffs(peers) - 1;
         uint32_t old = 0;
         if (lane == leader) old = atomicAdd(&warp_hist[warp][dg], (uint32_t)__popc(peers));
@@ -169,8 +194,12 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     }
     __syncthreads();
 
-    // offsets of each warp's run inside the digit, digit scan inside the tile
-    {
+    // offsets of each warp's run inside the digit, digit scan inside the tile (digits in order:
+    // all of q = 0 first, then q = 1)
+    uint32_t incl[DPT];
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = q * kRsThreads + threadIdx.x;
         uint32_t run = 0;
 #pragma unroll
         for (int w = 0; w < kRsWarps; ++w) {
@@ -178,85 +207,131 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
             warp_hist[w][d] = run;
             run += c;
         }
-    }
-    uint32_t incl = count;
+        incl[q] = count[q];
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        uint32_t v = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += v;
+        for (int off = 1; off < 32; off <<= 1) {
+            uint32_t v = __shfl_up_sync(0xffffffffu, incl[q], off);
+            if (lane >= off) incl[q] += v;
+        }
+        if (lane == 31) warp_tot[q][warp] = incl[q];
     }
-    if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    uint32_t wbase = 0;
-    for (int w = 0; w < warp; ++w) wbase += warp_tot[w];
-    const uint32_t excl_in_tile = wbase + incl - count;
-    digit_excl[d] = excl_in_tile;
+    uint32_t excl[DPT];
+    {
+        uint32_t carry = 0;
+#pragma unroll
+        for (int q = 0; q < DPT; ++q) {
+            uint32_t wbase = 0, total = 0;
+#pragma unroll
+            for (int w = 0; w < kRsWarps; ++w) {
+                const uint32_t c = warp_tot[q][w];
+                if (w < warp) wbase += c;
+                total += c;
+            }
+            excl[q] = carry + wbase + incl[q] - count[q];
+            digit_excl[q * kRsThreads + threadIdx.x] = excl[q];
+            carry += total;
+        }
+    }
     __syncthreads();
 
     // Reorder in shared memory first (the payload is fetched only now: it is not needed for ranking).
     // This needs tile-local offsets only, so it runs before the look-back: by the time the global
     // prefix is needed, most predecessors have published theirs and little time is spent polling.
+    {
+        const V *vtile = vin + tile_base + mine;
 #pragma unroll
-    for (int i = 0; i < kRsItems; ++i) {
-        const int64_t idx = tile_base + warp * (32 * kRsItems) + i * 32 + lane;
-        const V val = idx < n ? vin[idx] : V(0);
-        const unsigned dg = (unsigned)(key[i] >> shift) & 255u;
-        const int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
-        keybuf[p] = key[i];
-        valbuf[p] = val;
+        for (int i = 0; i < kRsItems; ++i) {
+            const V val = mine + i * 32 < nvalid ? vtile[i * 32] : V(0);
+            const unsigned dg = (unsigned)(key[i] >> shift) & kDigitMask;
+            const int p = (int)digit_excl[dg] + (int)warp_hist[warp][dg] + rank[i];
+            keybuf[p] = key[i];
+            valbuf[p] = val;
+        }
     }
 
-    // chained scan over tiles (decoupled look-back); every wait is bounded
-    unsigned long long before = 0;
-    if (tile > 0) {
-        // The states of kLook predecessors are requested together, so a walk over tiles that have
-        // only published their own counts costs one memory round trip per kLook tiles.
-        constexpr int kLook = 8;
-        bool ok = true, done = false;
-        int64_t t = tile - 1;
-        while (ok && !done) {
-            unsigned long long s[kLook];
+    // Chained scan over tiles (decoupled look-back); every wait is bounded.  Most predecessors met
+    // on the way have published only their own counts, so those are taken kLook at a time with one
+    // test; a tile that is not ready yet, or one that carries a prefix, is handled one by one.
+    const unsigned tag_own = (epoch << 2) | kFlagOwn, tag_prefix = (epoch << 2) | kFlagPrefix;
+    bool ok = true;
 #pragma unroll
-            for (int b = 0; b < kLook; ++b) s[b] = t - b >= 0 ? st[(t - b) * kRsBins + d] : 0ull;
+    for (int q = 0; q < DPT; ++q) {
+        const int d = q * kRsThreads + threadIdx.x;
+        uint32_t before = 0;
+        if (tile > 0) {
+            constexpr int kLook = 8;
+            volatile unsigned long long *p = st + (size_t)(tile - 1) * kBins + d;   // nearest tile not yet added
+            uint32_t togo = tile;                                                    // tiles from p down to tile 0
+            bool done = false;
+            while (ok && !done) {
+                if (togo >= (uint32_t)kLook) {
+                    unsigned long long s[kLook];
 #pragma unroll
-            for (int b = 0; b < kLook; ++b) {
-                if (ok && !done && t - b >= 0) {
-                    unsigned long long v = s[b];
-                    int spins = 0;
-                    while (!((v >> 62) && ((v >> 32) & 0xffu) == epoch)) {
-                        if (++spins > kSpinLimit) { ok = false; break; }
-                        __nanosleep(spins < 8 ? 200 : 1000);   // back off at once: polling warps must not crowd the issue slots
-                        v = st[(t - b) * kRsBins + d];
+                    for (int b = 0; b < kLook; ++b) s[b] = *(p - (ptrdiff_t)b * kBins);
+                    bool all_own = true;
+                    uint32_t sum = 0;
+#pragma unroll
+                    for (int b = 0; b < kLook; ++b) {
+                        all_own = all_own && (unsigned)(s[b] >> 32) == tag_own;
+                        sum += (uint32_t)s[b];
                     }
-                    if (ok) {
-                        before += v & kValMask;
-                        if ((v >> 62) == 2ull || t - b == 0) done = true;
+                    if (all_own) {
+                        before += sum;
+                        p -= (ptrdiff_t)kLook * kBins;
+                        togo -= kLook;
+                        continue;
                     }
+                    // take the leading words that are ready; stop behind a prefix or at an unready one
+                    int taken = 0;
+                    bool stop = false;
+#pragma unroll
+                    for (int b = 0; b < kLook; ++b) {
+                        const unsigned h = (unsigned)(s[b] >> 32);
+                        if (!stop && (h == tag_own || h == tag_prefix)) {
+                            before += (uint32_t)s[b];
+                            ++taken;
+                            if (h == tag_prefix) { done = true; stop = true; }
+                        } else {
+                            stop = true;
+                        }
+                    }
+                    p -= (ptrdiff_t)taken * kBins;
+                    togo -= taken;
+                    if (done) break;
                 }
+                unsigned long long v = *p;
+                int spins = 0;
+                while ((unsigned)(v >> 32) != tag_own && (unsigned)(v >> 32) != tag_prefix) {
+                    if (++spins > kSpinLimit) { ok = false; break; }
+                    __nanosleep(spins < 8 ? 200 : 1000);   // back off at once: polling warps must not crowd the issue slots
+                    v = *p;
+                }
+                if (!ok) break;
+                before += (uint32_t)v;
+                done = (unsigned)(v >> 32) == tag_prefix;   // tile 0 always carries a prefix, so the walk ends there at the latest
+                p -= kBins;
+                --togo;
             }
-            t -= kLook;
+            if (ok) st[(size_t)tile * kBins + d] = status_word(epoch, kFlagPrefix, before + count[q]);
         }
-        if (ok) {
-            st[tile * kRsBins + d] = kFlagInc | tag | (before + count);
-        } else {
-            report(err, CONST_ERR_TIMEOUT);
-            s_abort = 1;
-        }
+        s_gbase[d] = digit_base[d] + before - excl[q];      // modulo 2^32; adding a tile-local position gives the true offset
     }
-    s_gbase[d] = (long long)digit_base[d] + (long long)before - (long long)excl_in_tile;
+    if (!ok) {
+        report(err, CONST_ERR_TIMEOUT);
+        s_abort = 1;
+    }
     __syncthreads();
     if (s_abort) return;
 
     // store runs of consecutive addresses
-    const int64_t left = n - tile_base;
-    const int nvalid = left < kRsTile ? (int)left : kRsTile;
 #pragma unroll
     for (int m = 0; m < kRsItems; ++m) {
-        int p = threadIdx.x + m * kRsThreads;
+        const int p = threadIdx.x + m * kRsThreads;
         if (p < nvalid) {
-            uint64_t k = keybuf[p];
-            unsigned dg = (unsigned)(k >> shift) & 255u;
-            long long o = s_gbase[dg] + p;
+            const uint64_t k = keybuf[p];
+            const unsigned dg = (unsigned)(k >> shift) & kDigitMask;
+            const uint32_t o = s_gbase[dg] + (uint32_t)p;
             kout[o] = k;
             vout[o] = valbuf[p];
         }
@@ -595,51 +670,81 @@ struct Scratch {            // stream-ordered temporaries of one build
 // Small buffers of one sort.  `zeroed` covers hist, counters, totals and the status word in one
 // allocation so that a single memset clears them.
 struct SortBufs {
-    uint32_t *hist;                    // [kMaxPasses][256] digit counts, then exclusive digit offsets
+    uint32_t *hist;                    // [kMaxPasses][kRsMaxBins] digit counts, then exclusive digit offsets
     uint32_t *counters;                // [kMaxPasses] tile tickets
-    unsigned long long *tile_status;   // [ntiles][256]
+    unsigned long long *tile_status;   // [ntiles][kRsMaxBins]
 };
 
-template <typename V>
-const_status_t sort_passes(uint64_t *&keys, uint64_t *&keys_alt, V *&vals, V *&vals_alt, int64_t n, int passes,
-                           const SortBufs &b, int32_t *status, cudaStream_t stream) {
-    if (n == 0 || passes == 0) return CONST_OK;
+template <typename V, int BITS>
+const_status_t launch_onesweep(const uint64_t *kin, uint64_t *kout, const V *vin, V *vout, int64_t n, int shift,
+                               const uint32_t *digit_base, const SortBufs &b, uint32_t *counter, int32_t *status,
+                               unsigned epoch, cudaStream_t stream) {
     const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
-    CB_CUDA(cudaMemsetAsync(b.tile_status, 0, sizeof(unsigned long long) * ntiles * kRsBins, stream));
-    CB_LAUNCH("rs_scan_hist", stream, rs_scan_hist<<<passes, 256, 0, stream>>>(b.hist));
     const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
     static bool attr_set[64] = {false};    // per template instance and device
     int dev = 0;
     CB_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+        CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    for (int p = 0; p < passes; ++p) {
-        CB_LAUNCH("rs_onesweep", stream,
-                  rs_onesweep<V><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(
-                      keys, keys_alt, vals, vals_alt, n, 8 * p, b.hist + p * kRsBins, b.tile_status, b.counters + p,
-                      status, (unsigned)(p + 1)));
+    CB_LAUNCH("rs_onesweep", stream,
+              rs_onesweep<V, BITS><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(
+                  kin, kout, vin, vout, n, shift, digit_base, b.tile_status, counter, status, epoch));
+    return CONST_OK;
+}
+
+// Sorts (keys, payload) by key.  The first pass reads the payload from `vals_src` (the caller's
+// array, never written); later passes alternate between vals_a and vals_b.  On return `keys` and
+// `vals_sorted` name the buffers that hold the result.
+template <typename V>
+const_status_t sort_passes(uint64_t *&keys, uint64_t *&keys_alt, const V *vals_src, V *vals_a, V *vals_b,
+                           V *&vals_sorted, int64_t n, const DigitPlan &dp, const SortBufs &b, int32_t *status,
+                           cudaStream_t stream) {
+    vals_sorted = vals_a;
+    if (n == 0) return CONST_OK;
+    if (dp.passes == 0) {
+        CB_CUDA(cudaMemcpyAsync(vals_a, vals_src, sizeof(V) * n, cudaMemcpyDeviceToDevice, stream));
+        return CONST_OK;
+    }
+    const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
+    CB_CUDA(cudaMemsetAsync(b.tile_status, 0, sizeof(unsigned long long) * ntiles * kRsMaxBins, stream));
+    CB_LAUNCH("rs_scan_hist", stream, rs_scan_hist<<<dp.passes, 256, 0, stream>>>(b.hist));
+    const V *vin = vals_src;
+    V *vout = vals_a;
+    for (int p = 0; p < dp.passes; ++p) {
+        const_status_t s = dp.bits[p] > 8
+            ? launch_onesweep<V, 9>(keys, keys_alt, vin, vout, n, dp.shift[p], b.hist + p * kRsMaxBins, b, b.counters + p,
+                                    status, (unsigned)(p + 1), stream)
+            : launch_onesweep<V, 8>(keys, keys_alt, vin, vout, n, dp.shift[p], b.hist + p * kRsMaxBins, b, b.counters + p,
+                                    status, (unsigned)(p + 1), stream);
+        if (s != CONST_OK) return s;
         std::swap(keys, keys_alt);
-        std::swap(vals, vals_alt);
+        vals_sorted = vout;
+        vin = vout;
+        vout = vout == vals_a ? vals_b : vals_a;
     }
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }
 
 // Everything between "keys packed" and "level sizes known": sort, flag counts, block scan.
-const_status_t sort_and_count(uint64_t *&keys, uint64_t *&keys_alt, void *&vals, void *&vals_alt, int64_t nnz,
-                              int passes, const_dtype_t dtype, const SortBufs &b, const LevelShifts &ls,
-                              uint32_t *block_counts, uint32_t *totals, int32_t *status, cudaStream_t stream) {
+const_status_t sort_and_count(uint64_t *&keys, uint64_t *&keys_alt, const void *vals_src, void *vals_a, void *vals_b,
+                              void *&vals_sorted, int64_t nnz, const DigitPlan &dp, const_dtype_t dtype,
+                              const SortBufs &b, const LevelShifts &ls, uint32_t *block_counts, uint32_t *totals,
+                              int32_t *status, cudaStream_t stream) {
     const_status_t s;
     if (dtype == CONST_F32) {
-        uint32_t *v = (uint32_t *)vals, *va = (uint32_t *)vals_alt;
-        s = sort_passes<uint32_t>(keys, keys_alt, v, va, nnz, passes, b, status, stream);
-        vals = v; vals_alt = va;
+        uint32_t *out = nullptr;
+        s = sort_passes<uint32_t>(keys, keys_alt, (const uint32_t *)vals_src, (uint32_t *)vals_a, (uint32_t *)vals_b, out,
+                                  nnz, dp, b, status, stream);
+        vals_sorted = out;
     } else {
-        unsigned long long *v = (unsigned long long *)vals, *va = (unsigned long long *)vals_alt;
-        s = sort_passes<unsigned long long>(keys, keys_alt, v, va, nnz, passes, b, status, stream);
-        vals = v; vals_alt = va;
+        unsigned long long *out = nullptr;
+        s = sort_passes<unsigned long long>(keys, keys_alt, (const unsigned long long *)vals_src,
+                                            (unsigned long long *)vals_a, (unsigned long long *)vals_b, out, nnz, dp, b,
+                                            status, stream);
+        vals_sorted = out;
     }
     if (s != CONST_OK) return s;
     const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
@@ -648,7 +753,25 @@ const_status_t sort_and_count(uint64_t *&keys, uint64_t *&keys_alt, void *&vals,
     return CONST_OK;
 }
 
-struct KeyLayout { int bits[kMaxOrder]; int shift[kMaxOrder]; int total_bits; int passes; };
+struct KeyLayout { int bits[kMaxOrder]; int shift[kMaxOrder]; int total_bits; DigitPlan digits; };
+
+// Fewest passes with 8- or 9-bit digits: every pass is 8 bits wide unless 9-bit passes are needed to
+// cover the key in that number of passes (43 bits -> 9 9 9 8 8).  A digit may reach past the top of
+// the key; those bits are zero.
+DigitPlan digit_plan(int total_bits) {
+    DigitPlan dp;
+    for (int p = 0; p < kMaxPasses; ++p) dp.shift[p] = dp.bits[p] = 0;
+    const int p8 = (total_bits + 7) / 8, p9 = (total_bits + kRsMaxBits - 1) / kRsMaxBits;
+    dp.passes = p9 < p8 ? p9 : p8;
+    const int wide = std::max(0, total_bits - 8 * dp.passes);      // passes that must take 9 bits
+    int acc = 0;
+    for (int p = 0; p < dp.passes; ++p) {
+        dp.bits[p] = p < wide ? kRsMaxBits : 8;
+        dp.shift[p] = acc;
+        acc += dp.bits[p];
+    }
+    return dp;
+}
 
 bool key_layout(int order, const int64_t *dims, const int *mode_order, KeyLayout &k) {
     k.total_bits = 0;
@@ -657,7 +780,7 @@ bool key_layout(int order, const int64_t *dims, const int *mode_order, KeyLayout
     if (k.total_bits > 64) return false;
     int acc = 0;
     for (int l = order - 1; l >= 0; --l) { k.shift[l] = acc; acc += k.bits[l]; }
-    k.passes = (k.total_bits + 7) / 8;
+    k.digits = digit_plan(k.total_bits);
     return true;
 }
 
@@ -752,13 +875,13 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
     {
         Scratch tmp(stream);
         uint64_t *keys = nullptr, *keys_alt = nullptr;
-        void *vals = nullptr, *vals_alt = nullptr;
+        void *vals = nullptr, *vals_alt = nullptr, *vals_sorted = nullptr;
         unsigned char *small = nullptr;          // hist | counters | totals | status, cleared together
         uint32_t *block_counts = nullptr;
         SortBufs sb{nullptr, nullptr, nullptr};
         const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
         const int64_t ntiles = (nnz + kRsTile - 1) / kRsTile;
-        constexpr size_t kHistBytes = sizeof(uint32_t) * kMaxPasses * kRsBins;
+        constexpr size_t kHistBytes = sizeof(uint32_t) * kMaxPasses * kRsMaxBins;
         constexpr size_t kSmallBytes = kHistBytes + 256;
         auto body = [&]() -> const_status_t {
             CB_CUDA(tmp.alloc((void **)&keys, sizeof(uint64_t) * nnz));
@@ -766,7 +889,7 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             CB_CUDA(tmp.alloc(&vals, vsize * (nnz + 4)));
             CB_CUDA(tmp.alloc(&vals_alt, vsize * (nnz + 4)));
             CB_CUDA(tmp.alloc((void **)&small, kSmallBytes));
-            CB_CUDA(tmp.alloc((void **)&sb.tile_status, sizeof(unsigned long long) * std::max<int64_t>(ntiles, 1) * kRsBins));
+            CB_CUDA(tmp.alloc((void **)&sb.tile_status, sizeof(unsigned long long) * std::max<int64_t>(ntiles, 1) * kRsMaxBins));
             CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * kCpLevels * std::max<int64_t>(cp_blocks, 1)));
             CB_CUDA(cudaMemsetAsync(small, 0, kSmallBytes, stream));
             sb.hist = reinterpret_cast<uint32_t *>(small);
@@ -778,10 +901,9 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = kl.shift[l];
             if (nnz > 0) {
                 PackArgs pa = pack_args(order, dims, mode_order, coords_dev, kl);
-                CB_LAUNCH("pack_hist", stream, launch_pack_hist(pa, nnz, kl.passes, keys, sb.hist, status, stream));
-                CB_CUDA(cudaMemcpyAsync(vals, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
-                const_status_t s = sort_and_count(keys, keys_alt, vals, vals_alt, nnz, kl.passes, dtype, sb, ls,
-                                                  block_counts, totals, status, stream);
+                CB_LAUNCH("pack_hist", stream, launch_pack_hist(pa, nnz, kl.digits, keys, sb.hist, status, stream));
+                const_status_t s = sort_and_count(keys, keys_alt, vals_dev, vals, vals_alt, vals_sorted, nnz, kl.digits,
+                                                  dtype, sb, ls, block_counts, totals, status, stream);
                 if (s != CONST_OK) return s;
             }
             uint32_t h_small[32] = {0};          // totals at [0..4), status at [16]
@@ -806,8 +928,9 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             sz.order = order;
             for (int l = 0; l < kMaxOrder; ++l) sz.n[l] = csf->n[l];
             CB_LAUNCH("csf_finish", stream, csf_finish<<<1, 32, 0, stream>>>(arr, sz));
-            csf->vals = vals;                 // the sorted payload buffer becomes the leaf value array
-            tmp.forget(vals);
+            if (!vals_sorted) vals_sorted = vals;
+            csf->vals = vals_sorted;          // the sorted payload buffer becomes the leaf value array
+            tmp.forget(vals_sorted);
 
             // per-slice leaf offsets and the default work lists
             const int64_t n0 = csf->n[0];
@@ -845,8 +968,8 @@ constexpr size_t kNaOffKeys0 = 0;
 constexpr size_t kNaOffKeys1 = kNaOffKeys0 + kNaKeys;
 constexpr size_t kNaOffVals = kNaOffKeys1 + kNaKeys;                      // second payload buffer (the first is the caller's output)
 constexpr size_t kNaOffTileStatus = kNaOffVals + kNaKeys;
-constexpr size_t kNaOffHist = kNaOffTileStatus + sizeof(unsigned long long) * kNaTiles * kRsBins;
-constexpr size_t kNaHistBytes = sizeof(uint32_t) * kMaxPasses * kRsBins;
+constexpr size_t kNaOffHist = kNaOffTileStatus + sizeof(unsigned long long) * kNaTiles * kRsMaxBins;
+constexpr size_t kNaHistBytes = sizeof(uint32_t) * kMaxPasses * kRsMaxBins;
 constexpr size_t kNaOffSmall = kNaOffHist + kNaHistBytes;                 // pass counters, level totals, status word
 constexpr size_t kNaSmallBytes = 256;
 constexpr size_t kNaOffBlockCounts = kNaOffSmall + kNaSmallBytes;
@@ -903,14 +1026,15 @@ const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nn
     for (int l = 0; l < kMaxOrder; ++l) ls.shift[l] = kl.shift[l];
     if (nnz > 0) {
         PackArgs pa = pack_args(order, dims, mode_order, coords_dev, kl);
-        launch_pack_hist(pa, nnz, kl.passes, keys, sb.hist, status, stream);
-        // the payload ping-pongs between the caller's output and the static buffer; start on the side
+        launch_pack_hist(pa, nnz, kl.digits, keys, sb.hist, status, stream);
+        // the payload alternates between the caller's output and the static buffer; start on the side
         // that makes the last pass land in the caller's output
-        void *first = (kl.passes % 2 == 0) ? vals_out : (void *)(base + kNaOffVals);
-        void *second = (kl.passes % 2 == 0) ? (void *)(base + kNaOffVals) : vals_out;
-        CB_CUDA(cudaMemcpyAsync(first, vals_dev, vsize * nnz, cudaMemcpyDeviceToDevice, stream));
-        rc = sort_and_count(keys, keys_alt, first, second, nnz, kl.passes, dtype, sb, ls, block_counts, totals, status,
-                            stream);
+        const bool odd = kl.digits.passes % 2 == 1 || kl.digits.passes == 0;
+        void *first = odd ? vals_out : (void *)(base + kNaOffVals);
+        void *second = odd ? (void *)(base + kNaOffVals) : vals_out;
+        void *sorted = nullptr;
+        rc = sort_and_count(keys, keys_alt, vals_dev, first, second, sorted, nnz, kl.digits, dtype, sb, ls, block_counts,
+                            totals, status, stream);
         if (rc != CONST_OK) return rc;
     }
     uint32_t h_small[32] = {0};                   // totals at [0..4), status at [16]

@@ -37,6 +37,18 @@ def test_several_tiles_and_ragged_tail(nnz):
         assert_csf_equal(h, op, mo)
 
 
+@pytest.mark.parametrize("dims,nnz", [((512, 512, 512), 250_003),      # 27 key bits: three 9-bit digits
+                                      ((512, 256), 100_000),           # 17 bits: one 9-bit and one 8-bit digit
+                                      ((2048, 2048, 2048, 512), 70_001),   # 42 bits: 9 9 8 8 8
+                                      ((3, 2, 2), 12)])                # 5 bits: one short digit
+def test_digit_widths(dims, nnz):
+    rng = np.random.default_rng(sum(dims) + nnz)
+    for dtype in (np.float32, np.float64):
+        op = random_op(rng, dims, nnz, dtype=dtype)
+        mo = tuple(reversed(range(len(dims))))
+        assert_csf_equal(build_csf(op, mo), op, mo)
+
+
 def test_order4_wide_key_and_fp64_values():
     rng = np.random.default_rng(5)
     op = random_op(rng, (20000, 20000, 20000, 20000), 60_000)        # 60-bit key, 8 passes
