@@ -10,19 +10,27 @@
 //
 // Tiling.  T_i (n_k x n_l doubles, 1 MiB at the benchmark size) does not fit on chip, so a block
 // owns a strip of IS consecutive i slices and a tile of LT consecutive l values and keeps
-// T[LT][n_k][IS] in shared memory.  Strip-mining i lets every W nonzero fetched from L2 serve IS
-// rows of Z; tiling l does not change the result because Z is a sum over l.  With l at the root of
-// W, the nonzeros a block needs form one contiguous range of W's fibres.  The partial sums of the
-// (l, m) fibres are combined with fp64 atomic adds on Z.
+// T[LT][n_k][IS] in shared memory.  Strip-mining i lets every W nonzero fetched serve IS rows of Z;
+// tiling l does not change the result because Z is a sum over l.  With l at the root of W, the
+// nonzeros a block needs form one contiguous range of W's fibres.
+//
+// Memory access.  A thread that walks its own fibre straight from global memory touches a
+// different cache line than every other lane of its warp at every step, and the L1 tag stage
+// becomes the limit.  So both phases sweep their fibre range in chunks: the chunk's (coordinate,
+// value) pairs are copied into shared memory with coalesced loads as 16-byte records, and a group
+// of GL lanes then walks one fibre, every lane of the group reading the same record (one broadcast
+// 128-bit shared-memory load) and its own VPT = 8/GL entries of the V row (producer, contiguous
+// in global memory) or of the T row (consumer, contiguous in shared memory).  The partial sums of
+// the (l, m) fibres are combined with fp64 atomic adds on Z.
 #include "common.cuh"
 
 namespace cb {
 namespace {
 
-constexpr int IS = 8;      // i slices per block
-constexpr int LT = 8;      // l values per block
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+constexpr int LT = 8;          // l values per block
+constexpr int kThreads = 512;
+constexpr int RB = 2048;       // records staged per chunk
+constexpr int FPMAX = 1024;    // fibre descriptors staged per batch
 
 struct Csf3d {
     const int32_t *crd0, *pos1, *crd1, *pos2, *crd2;
@@ -30,18 +38,86 @@ struct Csf3d {
     int32_t n0;
 };
 
+struct __align__(16) Rec {
+    int32_t c;
+    int32_t pad;
+    double v;
+};
+
+struct Stage {                 // shared-memory staging area of one sweep
+    Rec *recs;                 // [RB]
+    int32_t *fpos;             // [FPMAX + 1] first nonzero of every staged fibre
+    int32_t *fcrd;             // [FPMAX]     level-1 coordinate of every staged fibre
+};
+
+// Calls body(fibre, coordinate, records, count) once for every piece of every fibre in [fA, fB) of
+// the tensor x; a fibre that straddles a chunk boundary is delivered in two pieces (in different
+// chunks, i.e. separated by a block barrier).  Lane groups take the fibres of a chunk round-robin.
+template <int GL, class Body>
+__device__ __forceinline__ void sweep(const Csf3d &x, int32_t fA, int32_t fB, const Stage &st, Body body) {
+    constexpr int NG = kThreads / GL;
+    const int g = threadIdx.x / GL;
+    for (int32_t fb0 = fA; fb0 < fB; fb0 += FPMAX) {
+        const int nf = fB - fb0 < FPMAX ? fB - fb0 : FPMAX;
+        __syncthreads();
+        for (int e = threadIdx.x; e <= nf; e += kThreads) st.fpos[e] = __ldg(x.pos2 + fb0 + e);
+        for (int e = threadIdx.x; e < nf; e += kThreads) st.fcrd[e] = __ldg(x.crd1 + fb0 + e);
+        __syncthreads();
+        const int32_t pA = st.fpos[0], pB = st.fpos[nf];
+        for (int32_t c0 = pA; c0 < pB; c0 += RB) {
+            const int32_t c1 = c0 + RB < pB ? c0 + RB : pB;
+            for (int e = threadIdx.x; e < c1 - c0; e += kThreads) {
+                Rec r;
+                r.c = __ldg(x.crd2 + c0 + e);
+                r.pad = 0;
+                r.v = __ldg(x.vals + c0 + e);
+                st.recs[e] = r;
+            }
+            __syncthreads();
+            int lo = 0, hi = nf - 1;                       // staged fibre that holds nonzero c0
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (st.fpos[mid] <= c0) lo = mid; else hi = mid - 1;
+            }
+            for (int f = lo + g; f < nf; f += NG) {
+                const int32_t a = st.fpos[f], b = st.fpos[f + 1];
+                if (a >= c1) break;
+                const int32_t p0 = a > c0 ? a : c0, p1 = b < c1 ? b : c1;
+                if (p0 < p1) body(fb0 + f, st.fcrd[f], st.recs + (p0 - c0), p1 - p0);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+template <int IS, int GL>
 __global__ void __launch_bounds__(kThreads)
-network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restrict__ Z, int n_k, int n_l, int n_m) {
-    extern __shared__ double T[];                  // [LT][KP][IS], KP = n_k + 1 (odd row pitch spreads the banks)
+network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restrict__ Z, int n_k, int n_l, int n_m,
+               int v_vec_ok) {
+    constexpr int VPT = 8 / GL;                    // entries of a V row (producer) or T row (consumer) per lane
+    static_assert(LT == 8 && IS == 8 && (VPT == 1 || VPT == 2), "a lane group covers the 8 l of the tile or the 8 i of the strip");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int TL = n_k * IS + 2;                   // doubles per l plane; the +2 staggers the banks of the 8 planes
+    double *T = reinterpret_cast<double *>(smem_raw);                               // [LT][n_k][IS]
+    Stage st;
+    st.recs = reinterpret_cast<Rec *>(T + ((size_t)LT * TL + 1) / 2 * 2);
+    st.fpos = reinterpret_cast<int32_t *>(st.recs + RB);
+    st.fcrd = st.fpos + FPMAX + 1;
+    __shared__ int32_t s_pos[IS + 1];              // first fibre of every slice of the strip
     __shared__ int32_t w_pos[LT + 1];              // first fibre of every l node of the tile
     __shared__ int32_t w_l[LT];                    // l of those nodes, relative to the tile
     __shared__ int32_t w_nodes;
-    const int KP = n_k + 1;
+
     const int strip = blockIdx.x, l0 = blockIdx.y * LT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int q = threadIdx.x % GL;                // position inside the lane group
 
-    for (int e = threadIdx.x; e < LT * KP * IS; e += kThreads) T[e] = 0.0;      // "T[*,*] = 0" per fused iteration
-    if (warp == 0) {
+    for (int e = threadIdx.x; e < LT * TL; e += kThreads) T[e] = 0.0;              // "T[*,*] = 0" per fused iteration
+    if (threadIdx.x <= IS) {
+        const int s = strip * IS + threadIdx.x;
+        s_pos[threadIdx.x] = __ldg(u.pos1 + (s < u.n0 ? s : u.n0));
+    }
+    if (warp == 1) {
         // root nodes of W whose l lies in [l0, l0 + LT): a contiguous range of at most LT nodes
         int32_t lo = 0, hi = w.n0;
         while (lo < hi) { int32_t mid = lo + (hi - lo) / 2; if (__ldg(w.crd0 + mid) < l0) lo = mid + 1; else hi = mid; }
@@ -54,115 +130,90 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
         if (lane == 0) { w_nodes = cnt; w_pos[cnt] = __ldg(w.pos1 + first + cnt); }
     }
     __syncthreads();
-
-    // ---- producer: T[l][k][ii] = sum_j U[i,k,j] * V[j, l0 + l]; LT/4 lanes per (i,k) fibre, four l per lane,
-    //      so every (j, value) pair fetched feeds four multiply-adds
-    {
-        constexpr int LPU = LT / 4;                // lanes per fibre
-        constexpr int UNITS = kThreads / LPU;      // fibres in flight per block
-        const int slot = threadIdx.x / LPU, l4 = (threadIdx.x % LPU) * 4;
-        const bool vec = (n_l % 2 == 0) && (l0 + l4 + 3 < n_l);     // 16-byte aligned, fully inside the row
-        const double *vcol = V + l0 + l4;
-        for (int ii = 0; ii < IS; ++ii) {
-            const int s = strip * IS + ii;
-            if (s >= u.n0) break;
-            const int32_t fa = __ldg(u.pos1 + s), fb = __ldg(u.pos1 + s + 1);
-            int32_t kn = 0, pan = 0, pbn = 0;                  // descriptor of the fibre after this one
-            if (fa + slot < fb) {
-                kn = __ldg(u.crd1 + fa + slot); pan = __ldg(u.pos2 + fa + slot); pbn = __ldg(u.pos2 + fa + slot + 1);
-            }
-            for (int32_t f = fa + slot; f < fb; f += UNITS) {
-                const int32_t k = kn, pa = pan, pb = pbn;
-                if (f + UNITS < fb) {
-                    kn = __ldg(u.crd1 + f + UNITS); pan = __ldg(u.pos2 + f + UNITS); pbn = __ldg(u.pos2 + f + UNITS + 1);
-                }
-                double a[4] = {0.0, 0.0, 0.0, 0.0};
-                if (vec) {
-                    int32_t p = pa;
-                    for (; p + 1 < pb; p += 2) {
-                        const int32_t j0 = __ldg(u.crd2 + p), j1 = __ldg(u.crd2 + p + 1);
-                        const double x0 = __ldg(u.vals + p), x1 = __ldg(u.vals + p + 1);
-                        const double2 *r0 = reinterpret_cast<const double2 *>(vcol + (size_t)j0 * n_l);
-                        const double2 *r1 = reinterpret_cast<const double2 *>(vcol + (size_t)j1 * n_l);
-                        const double2 v00 = __ldg(r0), v01 = __ldg(r0 + 1), v10 = __ldg(r1), v11 = __ldg(r1 + 1);
-                        a[0] = fma(x0, v00.x, a[0]); a[1] = fma(x0, v00.y, a[1]);
-                        a[2] = fma(x0, v01.x, a[2]); a[3] = fma(x0, v01.y, a[3]);
-                        a[0] = fma(x1, v10.x, a[0]); a[1] = fma(x1, v10.y, a[1]);
-                        a[2] = fma(x1, v11.x, a[2]); a[3] = fma(x1, v11.y, a[3]);
-                    }
-                    if (p < pb) {
-                        const double x0 = __ldg(u.vals + p);
-                        const double2 *r0 = reinterpret_cast<const double2 *>(vcol + (size_t)__ldg(u.crd2 + p) * n_l);
-                        const double2 v00 = __ldg(r0), v01 = __ldg(r0 + 1);
-                        a[0] = fma(x0, v00.x, a[0]); a[1] = fma(x0, v00.y, a[1]);
-                        a[2] = fma(x0, v01.x, a[2]); a[3] = fma(x0, v01.y, a[3]);
-                    }
-                } else {
-                    for (int32_t p = pa; p < pb; ++p) {
-                        const double x0 = __ldg(u.vals + p);
-                        const double *r0 = vcol + (size_t)__ldg(u.crd2 + p) * n_l;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            if (l0 + l4 + c < n_l) a[c] = fma(x0, __ldg(r0 + c), a[c]);
-                    }
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (l0 + l4 + c < n_l) T[((l4 + c) * KP + k) * IS + ii] = a[c];
-            }
-        }
-    }
-    __syncthreads();
-
-    // ---- consumer: two lanes (four i of the strip each) per (l, m) fibre of W, so every (k, value) pair
-    //      fetched feeds four multiply-adds and a warp has sixteen independent fibres in flight; the
-    //      descriptor of the next fibre is fetched ahead
-    constexpr int LPFIB = IS / 4;                               // lanes per fibre
-    constexpr int SLOTS = kThreads / LPFIB;
-    const int i4 = (threadIdx.x % LPFIB) * 4, slot = threadIdx.x / LPFIB;
-    int32_t rows[4];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const int s_row = strip * IS + i4 + c;
-        rows[c] = s_row < u.n0 ? __ldg(u.crd0 + s_row) : -1;
-    }
     const int nodes = w_nodes;
-    if (nodes == 0) return;
-    const int32_t f_begin = w_pos[0], f_end = w_pos[nodes];
-    int32_t f = f_begin + slot;
-    int32_t m = 0, pa = 0, pb = 0;
-    if (f < f_end) { m = __ldg(w.crd1 + f); pa = __ldg(w.pos2 + f); pb = __ldg(w.pos2 + f + 1); }
-    while (f < f_end) {
-        const int32_t fn = f + SLOTS;
-        int32_t mn = 0, pan = 0, pbn = 0;
-        if (fn < f_end) { mn = __ldg(w.crd1 + fn); pan = __ldg(w.pos2 + fn); pbn = __ldg(w.pos2 + fn + 1); }
-        int node = 0;
-        while (node + 1 < nodes && w_pos[node + 1] <= f) ++node;
-        const double *t = T + (size_t)w_l[node] * KP * IS + i4;
-        double a[4] = {0.0, 0.0, 0.0, 0.0};
-        int32_t p = pa;
-        for (; p + 1 < pb; p += 2) {
-            const int32_t k0 = __ldg(w.crd2 + p), k1 = __ldg(w.crd2 + p + 1);
-            const double w0 = __ldg(w.vals + p), w1 = __ldg(w.vals + p + 1);
-            const double2 *t0 = reinterpret_cast<const double2 *>(t + k0 * IS);
-            const double2 *t1 = reinterpret_cast<const double2 *>(t + k1 * IS);
-            const double2 t00 = t0[0], t01 = t0[1], t10 = t1[0], t11 = t1[1];
-            a[0] = fma(t00.x, w0, a[0]); a[1] = fma(t00.y, w0, a[1]);
-            a[2] = fma(t01.x, w0, a[2]); a[3] = fma(t01.y, w0, a[3]);
-            a[0] = fma(t10.x, w1, a[0]); a[1] = fma(t10.y, w1, a[1]);
-            a[2] = fma(t11.x, w1, a[2]); a[3] = fma(t11.y, w1, a[3]);
-        }
-        if (p < pb) {
-            const double w0 = __ldg(w.vals + p);
-            const double2 *t0 = reinterpret_cast<const double2 *>(t + __ldg(w.crd2 + p) * IS);
-            const double2 t00 = t0[0], t01 = t0[1];
-            a[0] = fma(t00.x, w0, a[0]); a[1] = fma(t00.y, w0, a[1]);
-            a[2] = fma(t01.x, w0, a[2]); a[3] = fma(t01.y, w0, a[3]);
-        }
+    if (nodes == 0) return;                        // no W nonzero has its l in this tile: nothing reaches Z
+
+    // ---- producer: T[l][k][ii] = sum_j U[i,k,j] * V[j, l0 + l]
+    {
+        const int lq = q * VPT;                    // first l of this lane, relative to the tile
+        const double *vcol = V + l0 + lq;
+        const bool full = l0 + lq + VPT <= n_l;
+        sweep<GL>(u, s_pos[0], s_pos[IS], st, [&](int32_t f, int32_t k, const Rec *recs, int n) {
+            int ii = 0;
+            while (ii + 1 < IS && s_pos[ii + 1] <= f) ++ii;
+            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
+            if (VPT == 2 && v_vec_ok && full) {
+                int e = 0;
+                for (; e + 1 < n; e += 2) {
+                    const Rec r0 = recs[e], r1 = recs[e + 1];
+                    const double2 v0 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r0.c * n_l));
+                    const double2 v1 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r1.c * n_l));
+                    a0 = fma(r0.v, v0.x, a0); a1 = fma(r0.v, v0.y, a1);
+                    b0 = fma(r1.v, v1.x, b0); b1 = fma(r1.v, v1.y, b1);
+                }
+                if (e < n) {
+                    const Rec r0 = recs[e];
+                    const double2 v0 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r0.c * n_l));
+                    a0 = fma(r0.v, v0.x, a0); a1 = fma(r0.v, v0.y, a1);
+                }
+                a0 += b0; a1 += b1;
+            } else {
+                for (int e = 0; e < n; ++e) {
+                    const Rec r0 = recs[e];
+                    const double *row = vcol + (size_t)r0.c * n_l;
+                    if (l0 + lq < n_l) a0 = fma(r0.v, __ldg(row), a0);
+                    if (VPT == 2 && l0 + lq + 1 < n_l) a1 = fma(r0.v, __ldg(row + 1), a1);
+                }
+            }
+            double *t = T + (size_t)lq * TL + k * IS + ii;
+            t[0] += a0;
+            if (VPT == 2) t[TL] += a1;
+        });
+    }
+    // (the sweep ends with a block barrier: T is complete)
+
+    // ---- consumer: Z[i,m] += sum_{k in fibre (l,m)} T[l][k][ii] * W[l,m,k]
+    {
+        const int iq = q * VPT;                    // first slice of this lane, relative to the strip
+        int32_t rows[VPT];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (rows[c] >= 0) atomicAdd(Z + (size_t)rows[c] * n_m + m, a[c]);
-        f = fn; m = mn; pa = pan; pb = pbn;
+        for (int c = 0; c < VPT; ++c) {
+            const int s = strip * IS + iq + c;
+            rows[c] = s < u.n0 ? __ldg(u.crd0 + s) : -1;
+        }
+        sweep<GL>(w, w_pos[0], w_pos[nodes], st, [&](int32_t f, int32_t m, const Rec *recs, int n) {
+            int node = 0;
+            while (node + 1 < nodes && w_pos[node + 1] <= f) ++node;
+            const double *t = T + (size_t)w_l[node] * TL + iq;
+            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
+            if (VPT == 2) {
+                int e = 0;
+                for (; e + 1 < n; e += 2) {
+                    const Rec r0 = recs[e], r1 = recs[e + 1];
+                    const double2 t0 = *reinterpret_cast<const double2 *>(t + r0.c * IS);
+                    const double2 t1 = *reinterpret_cast<const double2 *>(t + r1.c * IS);
+                    a0 = fma(t0.x, r0.v, a0); a1 = fma(t0.y, r0.v, a1);
+                    b0 = fma(t1.x, r1.v, b0); b1 = fma(t1.y, r1.v, b1);
+                }
+                if (e < n) {
+                    const Rec r0 = recs[e];
+                    const double2 t0 = *reinterpret_cast<const double2 *>(t + r0.c * IS);
+                    a0 = fma(t0.x, r0.v, a0); a1 = fma(t0.y, r0.v, a1);
+                }
+                a0 += b0; a1 += b1;
+            } else {
+                int e = 0;
+                for (; e + 1 < n; e += 2) {
+                    const Rec r0 = recs[e], r1 = recs[e + 1];
+                    a0 = fma(t[r0.c * IS], r0.v, a0);
+                    b0 = fma(t[r1.c * IS], r1.v, b0);
+                }
+                if (e < n) a0 = fma(t[recs[e].c * IS], recs[e].v, a0);
+                a0 += b0;
+            }
+            if (rows[0] >= 0) atomicAdd(Z + (size_t)rows[0] * n_m + m, a0);
+            if (VPT == 2 && rows[VPT - 1] >= 0) atomicAdd(Z + (size_t)rows[VPT - 1] * n_m + m, a1);
+        });
     }
 }
 
@@ -171,15 +222,20 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
 const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z, int64_t n_i,
                            int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m, int32_t *, cudaStream_t stream) {
     (void)n_j;
+    constexpr int IS = 8, GL = 4;
     CB_CUDA(cudaMemsetAsync(Z, 0, sizeof(double) * n_i * n_m, stream));
     if (U->nnz == 0 || W->nnz == 0) return CONST_OK;
-    const size_t smem = sizeof(double) * LT * (n_k + 1) * IS;
-    if (smem > 200 * 1024 || n_l > (1ll << 30) || n_m > (1ll << 30)) return CONST_ERR_WORKSPACE;
-    CB_CUDA(cudaFuncSetAttribute(network_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t t_doubles = ((size_t)LT * (n_k * IS + 2) + 1) / 2 * 2;
+    const size_t smem = sizeof(double) * t_doubles + sizeof(Rec) * RB + sizeof(int32_t) * (2 * FPMAX + 1);
+    if (smem > 220 * 1024 || n_l > (1ll << 30) || n_m > (1ll << 30)) return CONST_ERR_WORKSPACE;
+    auto kernel = network_kernel<IS, GL>;
+    CB_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     Csf3d u{U->crd[0], U->pos[1], U->crd[1], U->pos[2], U->crd[2], static_cast<const double *>(U->vals), (int32_t)U->n[0]};
     Csf3d w{W->crd[0], W->pos[1], W->crd[1], W->pos[2], W->crd[2], static_cast<const double *>(W->vals), (int32_t)W->n[0]};
+    const int v_vec_ok = (n_l % 2 == 0) && (reinterpret_cast<uintptr_t>(V) % 16 == 0);
     dim3 grid((unsigned)((U->n[0] + IS - 1) / IS), (unsigned)((n_l + LT - 1) / LT));
-    CB_LAUNCH("network_kernel", stream, network_kernel<<<grid, kThreads, smem, stream>>>(u, V, w, Z, (int)n_k, (int)n_l, (int)n_m));
+    CB_LAUNCH("network_kernel", stream,
+              kernel<<<grid, kThreads, smem, stream>>>(u, V, w, Z, (int)n_k, (int)n_l, (int)n_m, v_vec_ok));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }
