@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     const_schedule_check,
     const_plan_reduced_order,
     const_plan_family,
+    const_plan_set_tensor_stage,
     const_execute,
     const_last_device_status,
     const_destroy,

@@ -70,6 +70,8 @@ def load_library():
     lib.const_plan_family.restype = ctypes.c_char_p
     lib.const_execute.argtypes = [vp, pp(_Operand), i32, vp, vp]
     lib.const_last_device_status.argtypes = [vp, vp]
+    lib.const_plan_set_tensor_stage.argtypes = [vp, i32]
+    lib.const_plan_set_tensor_stage.restype = i32
     lib.const_destroy.argtypes = [vp]
     lib.const_destroy.restype = None
     lib.const_profile_enable.argtypes = [i32]
@@ -311,6 +313,10 @@ def const_execute(plan: PlanHandle, operands: Dict[str, Union[CsfHandle, "object
         raise ValueError("output must be a contiguous CUDA tensor")
     _check(lib.const_execute(plan.ptr, ops, len(operands), ctypes.c_void_p(out.data_ptr()), _stream_ptr(stream)),
            "const_execute")
+
+
+def const_plan_set_tensor_stage(plan: PlanHandle, enable: bool) -> None:
+    _check(load_library().const_plan_set_tensor_stage(plan.ptr, 1 if enable else 0), "const_plan_set_tensor_stage")
 
 
 def const_last_device_status(plan: PlanHandle, stream=None) -> int:

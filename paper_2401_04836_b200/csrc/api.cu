@@ -207,6 +207,9 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
             return run_mttkrp3(X, (const float *)dense[0], (const float *)dense[1], d.ranks[0], (float *)out_dev,
                                n_rows, p->status_dev, stream);
         case Family::Ttmc4:
+            if (p->tensor_stage)
+                return run_ttmc4_tensor(X, (const float *)dense[0], (const float *)dense[1], (const float *)dense[2],
+                                        d.ranks[0], (float *)out_dev, n_rows, p->status_dev, stream);
             return run_ttmc4(X, (const float *)dense[0], (const float *)dense[1], (const float *)dense[2], d.ranks[0],
                              (float *)out_dev, n_rows, p->status_dev, stream);
         case Family::Network: {
@@ -224,6 +227,14 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
         default:
             return CONST_ERR_UNSUPPORTED;
     }
+}
+
+const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
+    const_plan *p = const_cast<const_plan *>(as_plan(h));
+    if (!p) return CONST_ERR_INVALID_ARG;
+    if (enable && p->desc.family != Family::Ttmc4) return CONST_ERR_UNSUPPORTED;
+    p->tensor_stage = enable ? 1 : 0;
+    return CONST_OK;
 }
 
 const_status_t const_last_device_status(const_plan_t *h, void *stream) {

@@ -57,6 +57,7 @@ struct const_plan {
     uint32_t magic = cb::kPlanMagic;
     cb::PlanDesc desc;
     int32_t *status_dev = nullptr;     // device status word written by kernels
+    int tensor_stage = 0;              // run the dense per-slice stage on the tensor cores where a kernel has one
     int device = -1;
 };
 
@@ -103,6 +104,9 @@ const_status_t run_mttkrp3(const const_csf *X, const float *B, const float *C, i
                            int64_t n_rows, int32_t *status, cudaStream_t stream);
 const_status_t run_ttmc4(const const_csf *X, const float *U, const float *V, const float *W, int R, float *Y,
                          int64_t n_rows, int32_t *status, cudaStream_t stream);
+// ttmc4_tc_kernel.cu: the same contraction with the per-slice dense stage on the tensor cores
+const_status_t run_ttmc4_tensor(const const_csf *X, const float *U, const float *V, const float *W, int R, float *Y,
+                                int64_t n_rows, int32_t *status, cudaStream_t stream);
 // network_kernels.cu
 const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z,
                            int64_t n_i, int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m,

@@ -1,0 +1,474 @@
+// Fused order-4 TTMc with the dense per-slice stage on the tensor cores (tcgen05, accumulators in
+// tensor memory).  Same chain as ttmc4_kernel.cu (Fig. 4(b) structure, fused on i -> j -> k):
+//   P[c]   = sum_l X[i,j,k,l] W[l,c]      order-1 intermediate, reset per (i,j,k)
+//   Q[b,c] = sum_k V[k,b] P[c]            order-2 intermediate, reset per (i,j)
+//   Y[i,a,b,c] += U[j,a] Q[b,c]
+// The last statement, summed over the fibres of a slice, is the contraction
+//   Y_i[(b,c), a] = sum_f Q_f[(b,c)] * U[j_f, a]          M = 64, N = 8, K = fibres,
+// which one tcgen05.mma of kind::tf32 consumes eight fibres at a time.
+//
+// Producer (CUDA cores).  A warp works on windows of WF (i,j) fibres.  The level-2 nodes of a window
+// are dealt to NS = 8 streams of four lanes as equal contiguous runs; lane h of a stream keeps rows
+// b = 2h, 2h+1 of Q in registers.  When a stream's run leaves a fibre, or ends, the lanes park their
+// part of Q as one K slot of the A operand.  A fibre cut between two streams simply occupies two K
+// slots with the same j: the contraction is linear, so the pieces need not be merged.
+//
+// Operands in shared memory (no swizzle, K-major, as the shared-memory matrix descriptor defines it:
+// core matrices of 8 rows x 16 bytes, i.e. 8 values of m (or n) by 4 consecutive K slots):
+//   A[m, k] at (k / 8) * 2048 + ((k % 8) / 4) * 1024 + (m / 8) * 128 + (m % 8) * 16 + (k % 4) * 4   m = 8 b + c
+//   B[n, k] at (k / 4) * 144 + n * 16 + (k % 4) * 4                                                 n = a
+// (the 16 spare bytes per K quad of B stagger the banks for the lanes that write it).  K-major puts
+// four K slots of one m side by side, but a stream finishes one slot at a time, so the pieces are
+// parked as plain rows first and the warp transposes the window through registers, splitting on the way.
+// fp32 precision from tf32 products: every operand x is split into hi = tf32(x) (round to nearest)
+// and lo = x - hi, and the three products hi*hi, lo*hi, hi*lo are accumulated in fp32 in tensor
+// memory; the dropped lo*lo term and the truncation of lo are below 2^-20 relative per term.
+//
+// A block has four warps because a warp can read only its own quarter of the 128 tensor-memory
+// lanes (rows 16w..16w+15 of an M = 64 accumulator live in lanes 32w..32w+15).  Work items are
+// sized for kWarpsPerBlock warps, so a block takes kWarps / kWarpsPerBlock consecutive items; every
+// warp owns an 8-column accumulator and the epilogue adds the accumulators of an item's warps.
+// Every wait on an mbarrier is bounded; on a timeout the block records CONST_ERR_TIMEOUT in the
+// status word, stops issuing MMAs, skips its stores and still frees its tensor memory.
+#include "common.cuh"
+
+namespace cb {
+namespace {
+
+constexpr int R = 8;
+constexpr int TILE = R * R * R;   // floats of one output row (slice)
+constexpr int SL = 4;             // lanes per node stream
+constexpr int NS = 32 / SL;       // node streams per warp
+constexpr int WF = 16;            // (i,j) fibres per window
+constexpr int SLOTS = 24;         // K slots per window: at most WF + NS - 1 pieces, padded to a multiple of 8
+constexpr int KG = SLOTS / 8;
+constexpr int kWarps = 4;
+constexpr int kItemsPerBlock = kWarps / kWarpsPerBlock;
+constexpr int kTmemCols = 32;     // kWarps accumulators of 8 columns
+static_assert(WF + NS - 1 <= SLOTS && SLOTS <= 32 && SLOTS % 8 == 0, "one lane per slot when the B operand is written");
+
+constexpr int A_FLOATS = KG * 512;        // one A operand of a window: [KG][2 K quads][8 m groups][8 m][4 k]
+constexpr int B_QUAD = 36;                // floats per K quad of B: [8 n][4 k] + 4 spare
+constexpr int B_FLOATS = KG * 2 * B_QUAD;
+constexpr int RAW_ROW = 68;               // floats per parked piece (64 + 4 spare: staggers the banks)
+static_assert(SLOTS * RAW_ROW <= 2 * A_FLOATS, "pieces are parked in the space of the A operands");
+constexpr int WARP_FLOATS = 2 * A_FLOATS + 2 * B_FLOATS;
+constexpr int WARP_INTS = 96;             // Ps[WF + 1], Js[WF], Jslot[SLOTS]
+constexpr size_t kWarpBytes = (sizeof(float) * WARP_FLOATS + sizeof(int32_t) * WARP_INTS + 127) / 128 * 128;
+
+// instruction descriptor: D fp32, A and B tf32, both K-major, N = 8, M = 64
+constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((8u >> 3) << 17) | ((64u >> 4) << 24);
+
+struct Csf4 {
+    const int32_t *crd0, *pos1, *crd1, *pos2, *crd2, *pos3, *crd3;
+    const float *vals;
+};
+
+__device__ __forceinline__ float4 ldg4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+
+__device__ __forceinline__ int32_t leaf_of(const Csf4 &x, int32_t f1) { return __ldg(x.pos3 + __ldg(x.pos2 + f1)); }
+
+__device__ __forceinline__ int32_t lower_bound_leaf(const Csf4 &x, int32_t lo, int32_t hi, int64_t target) {
+    while (lo < hi) {
+        int32_t mid = lo + (hi - lo) / 2;
+        if ((int64_t)leaf_of(x, mid) < target) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float tf32_rn(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+__device__ __forceinline__ void split4(const float4 &x, float4 &hi, float4 &lo) {
+    hi = make_float4(tf32_rn(x.x), tf32_rn(x.y), tf32_rn(x.z), tf32_rn(x.w));
+    lo = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
+}
+
+// shared-memory matrix descriptor, no swizzle: start address, K-direction ("leading") and
+// MN-direction ("stride") byte offsets between core matrices, all in 16-byte units
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46);
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t mbar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(mbar) : "memory");
+}
+
+// true when the phase with the given parity has completed; gives up after a bounded number of polls
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
+    for (int it = 0; it < (1 << 20); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+struct NodeInfo { int32_t k, pa, pb, l; float xv; };      // one level-2 node and its first leaf
+
+__device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t n_end) {
+    NodeInfo r{0, 0, 0, 0, 0.f};
+    if (n < n_end) {
+        r.k = __ldg(x.crd2 + n);
+        r.pa = __ldg(x.pos3 + n);
+        r.pb = __ldg(x.pos3 + n + 1);
+        r.l = __ldg(x.crd3 + r.pa);
+        r.xv = __ldg(x.vals + r.pa);
+    }
+    return r;
+}
+
+// Produces the window of (i,j) fibres [s0, s0 + cnt): parks every piece of Q as a K slot of the A
+// operand (hi and lo parts), then writes the matching U rows as the B operand.  Returns the number
+// of K slots, padded to a multiple of 8 (padding slots are zero in A and B).  Raw is where the pieces
+// are parked before the transposition; it may overlap Ahi and Alo.
+__device__ __forceinline__ int produce_window(const Csf4 &x, const float *__restrict__ U, const float *__restrict__ V,
+                                              const float *__restrict__ W, int32_t s0, int cnt, int lane,
+                                              float *Ahi, float *Alo, float *__restrict__ Bhi,
+                                              float *__restrict__ Blo, float *Raw, int32_t *__restrict__ Ps, int32_t *__restrict__ Js,
+                                              int32_t *__restrict__ Jslot) {
+    const int st = lane / SL, h = lane % SL;
+    if (lane <= cnt) Ps[lane] = __ldg(x.pos2 + s0 + lane);
+    if (lane < cnt) Js[lane] = __ldg(x.crd1 + s0 + lane);
+    __syncwarp();
+
+    const int32_t N0 = Ps[0], N1 = Ps[cnt];
+    const int32_t per = (N1 - N0 + NS - 1) / NS;
+    const int32_t na = N0 + st * per;
+    const int32_t nb = na + per < N1 ? na + per : N1;
+    const bool active = na < nb;
+    int f = 0;
+    bool split = false;
+    if (active) {
+        int lo = 0, hi = cnt - 1;                                 // fibre holding node na
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (Ps[mid] <= na) lo = mid; else hi = mid - 1;
+        }
+        f = lo;
+        split = Ps[f] < na;                                       // fibre f was begun by the stream before
+    }
+    // K slot of a piece = its fibre + the number of cut fibres at or before this stream
+    const unsigned cuts = __ballot_sync(0xffffffffu, split && h == 0);
+    const int slot_off = __popc(cuts & ((2u << (st * SL)) - 1u));
+    const int nslots = cnt + __popc(cuts);
+
+    if (active) {
+        int32_t fend = Ps[f + 1];
+        float Q[2][R];
+#pragma unroll
+        for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
+
+        auto park = [&]() {                                       // rows b = 2h, 2h+1 of this piece, as they are
+            const int slot = f + slot_off;
+            float *dst = Raw + slot * RAW_ROW + 2 * h * R;
+#pragma unroll
+            for (int b2 = 0; b2 < 2; ++b2) {
+                *reinterpret_cast<float4 *>(dst + b2 * R) = make_float4(Q[b2][0], Q[b2][1], Q[b2][2], Q[b2][3]);
+                *reinterpret_cast<float4 *>(dst + b2 * R + 4) = make_float4(Q[b2][4], Q[b2][5], Q[b2][6], Q[b2][7]);
+            }
+            if (h == 0) Jslot[slot] = Js[f];
+        };
+
+        // software pipeline over the nodes of the run: descriptors two nodes ahead, rows one node ahead
+        NodeInfo cur = load_node(x, na, nb);
+        NodeInfo nxt = load_node(x, na + 1, nb);
+        float4 w0 = ldg4(W + (size_t)cur.l * R), w1 = ldg4(W + (size_t)cur.l * R + 4);
+        float2 vb = __ldg(reinterpret_cast<const float2 *>(V + (size_t)cur.k * R + 2 * h));
+        for (int32_t n = na; n < nb; ++n) {
+            const NodeInfo nn = load_node(x, n + 2, nb);
+            float4 w0n = w0, w1n = w1;
+            float2 vbn = vb;
+            if (n + 1 < nb) {
+                w0n = ldg4(W + (size_t)nxt.l * R);
+                w1n = ldg4(W + (size_t)nxt.l * R + 4);
+                vbn = __ldg(reinterpret_cast<const float2 *>(V + (size_t)nxt.k * R + 2 * h));
+            }
+            // P = sum over the node's leaves of X * W[l, :]
+            float P[R] = {cur.xv * w0.x, cur.xv * w0.y, cur.xv * w0.z, cur.xv * w0.w,
+                          cur.xv * w1.x, cur.xv * w1.y, cur.xv * w1.z, cur.xv * w1.w};
+            for (int32_t p = cur.pa + 1; p < cur.pb; ++p) {       // further leaves of the node (rare when sparse)
+                const float xv = __ldg(x.vals + p);
+                const float *w = W + (size_t)__ldg(x.crd3 + p) * R;
+                const float4 a0 = ldg4(w), a1 = ldg4(w + 4);
+                P[0] = fmaf(xv, a0.x, P[0]); P[1] = fmaf(xv, a0.y, P[1]);
+                P[2] = fmaf(xv, a0.z, P[2]); P[3] = fmaf(xv, a0.w, P[3]);
+                P[4] = fmaf(xv, a1.x, P[4]); P[5] = fmaf(xv, a1.y, P[5]);
+                P[6] = fmaf(xv, a1.z, P[6]); P[7] = fmaf(xv, a1.w, P[7]);
+            }
+#pragma unroll
+            for (int c = 0; c < R; ++c) {                         // Q[b, :] += V[k, b] * P[:]
+                Q[0][c] = fmaf(vb.x, P[c], Q[0][c]);
+                Q[1][c] = fmaf(vb.y, P[c], Q[1][c]);
+            }
+            if (n + 1 == fend) {                                  // the run leaves fibre f
+                park();
+#pragma unroll
+                for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
+                ++f;
+                fend = Ps[f + 1 <= cnt ? f + 1 : cnt];
+            }
+            cur = nxt; nxt = nn; w0 = w0n; w1 = w1n; vb = vbn;
+        }
+        if (f < cnt && nb > Ps[f]) park();                        // the run ends inside fibre f
+    }
+    __syncwarp();
+
+    // A operand: lane reads column m of four consecutive pieces (a K quad), splits, and writes 16 bytes
+    // of the hi and of the lo operand.  The pieces lie where the operands go, so the whole window is
+    // read into registers first.  Slots beyond nslots are padding and read as zero.
+    const int padded = (nslots + 7) & ~7;
+    {
+        constexpr int UNITS = SLOTS / 4 * 2;                      // (K quad, half of m) pairs per lane
+        float4 raw[UNITS];
+#pragma unroll
+        for (int u = 0; u < UNITS; ++u) {
+            const int quad = u >> 1, m = lane + 32 * (u & 1);
+            const float *src = Raw + (4 * quad) * RAW_ROW + m;
+            raw[u].x = 4 * quad + 0 < nslots ? src[0] : 0.f;
+            raw[u].y = 4 * quad + 1 < nslots ? src[RAW_ROW] : 0.f;
+            raw[u].z = 4 * quad + 2 < nslots ? src[2 * RAW_ROW] : 0.f;
+            raw[u].w = 4 * quad + 3 < nslots ? src[3 * RAW_ROW] : 0.f;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < UNITS; ++u) {
+            const int quad = u >> 1, m = lane + 32 * (u & 1);
+            if (4 * quad < padded) {
+                float4 hi4, lo4;
+                split4(raw[u], hi4, lo4);
+                const int off = (quad >> 1) * 512 + (quad & 1) * 256 + (m >> 3) * 32 + (m & 7) * 4;
+                *reinterpret_cast<float4 *>(Ahi + off) = hi4;
+                *reinterpret_cast<float4 *>(Alo + off) = lo4;
+            }
+        }
+    }
+    // B operand: one lane per K slot
+    const int slot = lane;
+    if (slot < padded) {
+        float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f), u1 = u0;
+        if (slot < nslots) {
+            const float *up = U + (size_t)Jslot[slot] * R;
+            u0 = ldg4(up);
+            u1 = ldg4(up + 4);
+        }
+        float4 h0, l0, h1, l1;
+        split4(u0, h0, l0);
+        split4(u1, h1, l1);
+        float *bh = Bhi + (slot >> 2) * B_QUAD + (slot & 3), *bl = Blo + (slot >> 2) * B_QUAD + (slot & 3);
+        bh[0] = h0.x; bh[4] = h0.y; bh[8] = h0.z; bh[12] = h0.w; bh[16] = h1.x; bh[20] = h1.y; bh[24] = h1.z; bh[28] = h1.w;
+        bl[0] = l0.x; bl[4] = l0.y; bl[8] = l0.z; bl[12] = l0.w; bl[16] = l1.x; bl[20] = l1.y; bl[24] = l1.z; bl[28] = l1.w;
+    }
+    return padded;
+}
+
+__global__ void __launch_bounds__(kWarps * 32)
+ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *__restrict__ light_list, Csf4 x,
+                const float *__restrict__ U, const float *__restrict__ V, const float *__restrict__ W,
+                float *__restrict__ out, int32_t *__restrict__ status) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t mbar_all[kWarps];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int32_t acc_row[kWarps];          // output row of every warp's accumulator, -1: none
+    __shared__ int32_t acc_used[kWarps];         // the warp issued at least one MMA
+    __shared__ int32_t item_kind[kItemsPerBlock];
+    __shared__ int32_t failed;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int item_slot = warp / kWarpsPerBlock, wl = warp % kWarpsPerBlock;
+    const int64_t item_idx = (int64_t)blockIdx.x * kItemsPerBlock + item_slot;
+    const bool have = item_idx < n_items;
+    WorkItem it{0, 0, 0, kItemLight};
+    if (have) it = items[item_idx];
+    const bool light = it.kind == kItemLight;
+
+    int32_t slice = it.slice, fa = 0, fb = 0;
+    if (light) {
+        if (wl < it.f0) {
+            slice = __ldg(light_list + it.slice + wl);
+            fa = __ldg(x.pos1 + slice);
+            fb = __ldg(x.pos1 + slice + 1);
+        }
+    } else {
+        const int64_t lo = leaf_of(x, it.f0), hi = leaf_of(x, it.f1);
+        fa = wl == 0 ? it.f0 : lower_bound_leaf(x, it.f0, it.f1, lo + (hi - lo) * wl / kWarpsPerBlock);
+        fb = wl == kWarpsPerBlock - 1
+                 ? it.f1
+                 : lower_bound_leaf(x, it.f0, it.f1, lo + (hi - lo) * (wl + 1) / kWarpsPerBlock);
+    }
+
+    const uint32_t mbar = smem_u32(&mbar_all[warp]);
+    if (lane == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar) : "memory");
+        acc_row[warp] = fa < fb ? __ldg(x.crd0 + slice) : -1;
+        acc_used[warp] = 0;
+        if (wl == 0) item_kind[item_slot] = it.kind;
+        if (warp == 0) failed = 0;
+    }
+    __syncwarp();
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t d_tmem = tmem_base + 8u * warp;
+
+    float *Ahi = reinterpret_cast<float *>(smem_raw + kWarpBytes * warp);
+    float *Alo = Ahi + A_FLOATS;
+    float *Bhi = Alo + A_FLOATS;
+    float *Blo = Bhi + B_FLOATS;
+    int32_t *Ps = reinterpret_cast<int32_t *>(Blo + B_FLOATS);
+    int32_t *Js = Ps + 32;
+    int32_t *Jslot = Js + 32;
+    const uint32_t ahi_s = smem_u32(Ahi), alo_s = smem_u32(Alo), bhi_s = smem_u32(Bhi), blo_s = smem_u32(Blo);
+
+    uint32_t parity = 0;
+    bool pending = false, ok = true, first = true;
+    for (int32_t s0 = fa; s0 < fb && ok; s0 += WF) {
+        const int cnt = fb - s0 < WF ? fb - s0 : WF;
+        if (pending) {                                            // the MMAs of the previous window still read the operands
+            bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+            done = __shfl_sync(0xffffffffu, done, 0);
+            parity ^= 1;
+            pending = false;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (!done) { ok = false; break; }
+        }
+        const int padded = produce_window(x, U, V, W, s0, cnt, lane, Ahi, Alo, Bhi, Blo, Ahi, Ps, Js, Jslot);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // operand stores -> visible to the tensor core
+        __syncwarp();
+        if (lane == 0) {
+            for (int kg = 0; kg < padded / 8; ++kg) {
+                const uint64_t a_hi = smem_desc(ahi_s + kg * 2048, 1024, 128), a_lo = smem_desc(alo_s + kg * 2048, 1024, 128);
+                const uint64_t b_hi = smem_desc(bhi_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
+                const uint64_t b_lo = smem_desc(blo_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
+                umma_tf32(d_tmem, a_hi, b_hi, (first && kg == 0) ? 0u : 1u);
+                umma_tf32(d_tmem, a_lo, b_hi, 1u);
+                umma_tf32(d_tmem, a_hi, b_lo, 1u);
+            }
+            umma_commit(mbar);
+            acc_used[warp] = 1;
+        }
+        pending = true;
+        first = false;
+        __syncwarp();
+    }
+    if (pending) {
+        bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+        done = __shfl_sync(0xffffffffu, done, 0);
+        if (!done) ok = false;
+    }
+    if (!ok && lane == 0) {
+        failed = 1;
+        atomicExch(status, (int32_t)CONST_ERR_TIMEOUT);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+    // ---- epilogue: warp w holds rows m = 16 w + lane (lane < 16) of every accumulator
+    if (!failed) {
+        uint32_t r[kWarps][R];
+#pragma unroll
+        for (int a = 0; a < kWarps; ++a) {
+            const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + 8u * a;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(r[a][0]), "=r"(r[a][1]), "=r"(r[a][2]), "=r"(r[a][3]), "=r"(r[a][4]), "=r"(r[a][5]),
+                           "=r"(r[a][6]), "=r"(r[a][7])
+                         : "r"(taddr));
+        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (lane < 16) {
+            const int m = 16 * warp + lane;
+#pragma unroll
+            for (int p = 0; p < kItemsPerBlock; ++p) {
+                const int kind = item_kind[p];
+                if (kind == kItemLight) {
+#pragma unroll
+                    for (int q = 0; q < kWarpsPerBlock; ++q) {
+                        const int a = p * kWarpsPerBlock + q;
+                        if (acc_row[a] >= 0 && acc_used[a]) {
+                            float *dst = out + (size_t)acc_row[a] * TILE + m;
+#pragma unroll
+                            for (int n = 0; n < R; ++n) dst[n * 64] = __uint_as_float(r[a][n]);
+                        }
+                    }
+                } else {
+                    float sum[R];
+                    int row = -1;
+#pragma unroll
+                    for (int n = 0; n < R; ++n) sum[n] = 0.f;
+#pragma unroll
+                    for (int q = 0; q < kWarpsPerBlock; ++q) {
+                        const int a = p * kWarpsPerBlock + q;
+                        if (acc_row[a] >= 0 && acc_used[a]) {
+                            row = acc_row[a];
+#pragma unroll
+                            for (int n = 0; n < R; ++n) sum[n] += __uint_as_float(r[a][n]);
+                        }
+                    }
+                    if (row >= 0) {
+                        float *dst = out + (size_t)row * TILE + m;
+                        if (kind == kItemBlock) {
+#pragma unroll
+                            for (int n = 0; n < R; ++n) dst[n * 64] = sum[n];
+                        } else {
+#pragma unroll
+                            for (int n = 0; n < R; ++n) atomicAdd(dst + n * 64, sum[n]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(kTmemCols) : "memory");
+}
+
+}  // namespace
+
+const_status_t run_ttmc4_tensor(const const_csf *X, const float *U, const float *V, const float *W, int rank, float *Y,
+                                int64_t n_rows, int32_t *status, cudaStream_t stream) {
+    if (rank != R) return CONST_ERR_UNSUPPORTED;
+    CB_CUDA(cudaMemsetAsync(Y, 0, sizeof(float) * TILE * n_rows, stream));
+    if (X->n_items == 0) return CONST_OK;
+    Csf4 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], X->pos[3], X->crd[3],
+           static_cast<const float *>(X->vals)};
+    constexpr size_t dyn = kWarpBytes * kWarps;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    CB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        CB_CUDA(cudaFuncSetAttribute(ttmc4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    const unsigned grid = (unsigned)((X->n_items + kItemsPerBlock - 1) / kItemsPerBlock);
+    CB_LAUNCH("ttmc4_tc_kernel", stream,
+              ttmc4_tc_kernel<<<grid, kWarps * 32, dyn, stream>>>(X->items, (int)X->n_items, X->light_list, x, U, V, W, Y, status));
+    CB_CUDA(cudaGetLastError());
+    return CONST_OK;
+}
+
+}  // namespace cb

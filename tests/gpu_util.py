@@ -37,7 +37,7 @@ def assert_csf_equal(h, op, mode_order):
     assert vals.dtype == ovals.dtype and vals.tobytes() == ovals.tobytes()
 
 
-def run_workload(w, bins=None, handles=None):
+def run_workload(w, bins=None, handles=None, tensor_stage=None):
     """Build CSF (unless given), create the plan, execute; returns (output ndarray, csf handles)."""
     dtype = cb.F32 if w.dtype == np.float32 else cb.F64
     if handles is None:
@@ -46,6 +46,8 @@ def run_workload(w, bins=None, handles=None):
         for h in handles.values():
             cb.const_csf_set_bins(h, *bins)
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, dtype)
+    if tensor_stage is not None:
+        cb.const_plan_set_tensor_stage(plan, tensor_stage)
     operands = dict(handles)
     operands.update({n: to_dev(a) for n, a in w.dense.items()})
     out = torch.full(w.out_shape, float("nan"), dtype=torch.float32 if dtype == cb.F32 else torch.float64,

@@ -17,8 +17,8 @@ ALL_GIANT = (1, 2, 700)
 MIXED = (300, 3000, 1500)
 
 
-def check(w, bins=None):
-    out, handles = run_workload(w, bins)
+def check(w, bins=None, tensor_stage=None):
+    out, handles = run_workload(w, bins, tensor_stage=tensor_stage)
     S, A = oracle(w)
     return assert_close(out, S, A, w.dtype), handles
 
@@ -84,6 +84,28 @@ def test_ttmc4_each_bin(bins):
 def test_ttmc4_sparse_like_the_benchmark():
     w = make_config(3, scale=0.004)             # 200k nonzeros in 20000^4: every (i,j,k) fibre has one leaf
     check(w)
+
+
+@pytest.mark.parametrize("bins", [None, ALL_LIGHT, ALL_HEAVY, ALL_GIANT, MIXED])
+def test_ttmc4_tensor_stage_each_bin(bins):
+    # the per-slice stage Y_i = U_J^T Q_J on the tensor cores (split tf32 operands) meets the fp32 tolerance
+    w = ttmc4_workload((300, 40, 30, 50), 80_000, 8, slice_s=1.0, value="pm1", config_id=3)
+    check(w, bins, tensor_stage=True)
+
+
+def test_ttmc4_tensor_stage_sparse_like_the_benchmark():
+    w = make_config(3, scale=0.004)
+    check(w, tensor_stage=True)
+    w = ttmc4_workload((7, 5, 3, 4), 60, 8, slice_s=1.0, value="pm1", config_id=3)      # a handful of tiny slices
+    check(w, tensor_stage=True)
+
+
+def test_tensor_stage_only_where_a_kernel_has_one():
+    w = make_config(1)
+    plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, cb.F32)
+    with pytest.raises(cb.ConstError):
+        cb.const_plan_set_tensor_stage(plan, True)
+    cb.const_plan_set_tensor_stage(plan, False)
 
 
 def test_scaled_configs_2_and_4():
