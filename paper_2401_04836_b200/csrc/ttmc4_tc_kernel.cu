@@ -7,19 +7,24 @@
 //   Y_i[(b,c), a] = sum_f Q_f[(b,c)] * U[j_f, a]          M = 64, N = 8, K = fibres,
 // which one tcgen05.mma of kind::tf32 consumes eight fibres at a time.
 //
-// Producer (CUDA cores).  A warp works on windows of WF (i,j) fibres.  The level-2 nodes of a window
-// are dealt to NS = 8 streams of four lanes as equal contiguous runs; lane h of a stream keeps rows
-// b = 2h, 2h+1 of Q in registers.  When a stream's run leaves a fibre, or ends, the lanes park their
-// part of Q as one K slot of the A operand.  A fibre cut between two streams simply occupies two K
-// slots with the same j: the contraction is linear, so the pieces need not be merged.
+// Producer (CUDA cores).  The level-2 nodes of a warp's fibre range are dealt to NS = 8 streams of
+// four lanes as equal contiguous runs, which the streams walk from end to end with node descriptors
+// two nodes and factor rows one node ahead; lane h of a stream keeps rows b = 2h, 2h+1 of Q in
+// registers.  When a stream's run leaves a fibre, or ends, its lanes park their part of Q, with the
+// fibre's j, as one piece.  The contraction is linear in Q, so a piece is simply one K slot: a fibre
+// cut between two streams occupies two slots with the same j and nothing has to be merged.  Every
+// stream owns C slots; when one of them is full the warp flushes all 8 C slots (empty ones as zeros).
 //
-// Operands in shared memory (no swizzle, K-major, as the shared-memory matrix descriptor defines it:
-// core matrices of 8 rows x 16 bytes, i.e. 8 values of m (or n) by 4 consecutive K slots):
+// Flush.  Operands in shared memory (no swizzle, K-major, as the shared-memory matrix descriptor
+// defines it: core matrices of 8 rows x 16 bytes, i.e. 8 values of m (or n) by 4 consecutive K slots):
 //   A[m, k] at (k / 8) * 2048 + ((k % 8) / 4) * 1024 + (m / 8) * 128 + (m % 8) * 16 + (k % 4) * 4   m = 8 b + c
 //   B[n, k] at (k / 4) * 144 + n * 16 + (k % 4) * 4                                                 n = a
 // (the 16 spare bytes per K quad of B stagger the banks for the lanes that write it).  K-major puts
-// four K slots of one m side by side, but a stream finishes one slot at a time, so the pieces are
-// parked as plain rows first and the warp transposes the window through registers, splitting on the way.
+// four K slots of one m side by side, while a stream finishes one slot at a time, so pieces are parked
+// as plain rows and the flush transposes them: a lane reads column m of four pieces, splits, and
+// stores 16 bytes of each operand.  One lane then issues three MMAs per group of eight slots and
+// commits them to the warp's mbarrier; the streams go on walking while the tensor core works, and
+// the next flush waits for that commit before it overwrites the operands.
 // fp32 precision from tf32 products: every operand x is split into hi = tf32(x) (round to nearest)
 // and lo = x - hi, and the three products hi*hi, lo*hi, hi*lo are accumulated in fp32 in tensor
 // memory; the dropped lo*lo term and the truncation of lo are below 2^-20 relative per term.
@@ -39,21 +44,20 @@ constexpr int R = 8;
 constexpr int TILE = R * R * R;   // floats of one output row (slice)
 constexpr int SL = 4;             // lanes per node stream
 constexpr int NS = 32 / SL;       // node streams per warp
-constexpr int WF = 16;            // (i,j) fibres per window
-constexpr int SLOTS = 24;         // K slots per window: at most WF + NS - 1 pieces, padded to a multiple of 8
-constexpr int KG = SLOTS / 8;
+constexpr int C = 2;              // K slots (parked pieces) per stream between two flushes
+constexpr int SLOTS = NS * C;     // K slots per flush
+constexpr int KG = SLOTS / 8;     // groups of eight slots = MMAs per operand pair
 constexpr int kWarps = 4;
 constexpr int kItemsPerBlock = kWarps / kWarpsPerBlock;
 constexpr int kTmemCols = 32;     // kWarps accumulators of 8 columns
-static_assert(WF + NS - 1 <= SLOTS && SLOTS <= 32 && SLOTS % 8 == 0, "one lane per slot when the B operand is written");
+static_assert(SLOTS % 8 == 0 && SLOTS <= 32, "one lane per slot when the B operand is written");
 
-constexpr int A_FLOATS = KG * 512;        // one A operand of a window: [KG][2 K quads][8 m groups][8 m][4 k]
+constexpr int A_FLOATS = KG * 512;        // one A operand: [KG][2 K quads][8 m groups][8 m][4 k]
 constexpr int B_QUAD = 36;                // floats per K quad of B: [8 n][4 k] + 4 spare
 constexpr int B_FLOATS = KG * 2 * B_QUAD;
 constexpr int RAW_ROW = 68;               // floats per parked piece (64 + 4 spare: staggers the banks)
-static_assert(SLOTS * RAW_ROW <= 2 * A_FLOATS, "pieces are parked in the space of the A operands");
-constexpr int WARP_FLOATS = 2 * A_FLOATS + 2 * B_FLOATS;
-constexpr int WARP_INTS = 96;             // Ps[WF + 1], Js[WF], Jslot[SLOTS]
+constexpr int WARP_FLOATS = 2 * A_FLOATS + 2 * B_FLOATS + SLOTS * RAW_ROW;
+constexpr int WARP_INTS = 32;             // Jslot[SLOTS]
 constexpr size_t kWarpBytes = (sizeof(float) * WARP_FLOATS + sizeof(int32_t) * WARP_INTS + 127) / 128 * 128;
 
 // instruction descriptor: D fp32, A and B tf32, both K-major, N = 8, M = 64
@@ -133,150 +137,6 @@ __device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t 
     return r;
 }
 
-// Produces the window of (i,j) fibres [s0, s0 + cnt): parks every piece of Q as a K slot of the A
-// operand (hi and lo parts), then writes the matching U rows as the B operand.  Returns the number
-// of K slots, padded to a multiple of 8 (padding slots are zero in A and B).  Raw is where the pieces
-// are parked before the transposition; it may overlap Ahi and Alo.
-__device__ __forceinline__ int produce_window(const Csf4 &x, const float *__restrict__ U, const float *__restrict__ V,
-                                              const float *__restrict__ W, int32_t s0, int cnt, int lane,
-                                              float *Ahi, float *Alo, float *__restrict__ Bhi,
-                                              float *__restrict__ Blo, float *Raw, int32_t *__restrict__ Ps, int32_t *__restrict__ Js,
-                                              int32_t *__restrict__ Jslot) {
-    const int st = lane / SL, h = lane % SL;
-    if (lane <= cnt) Ps[lane] = __ldg(x.pos2 + s0 + lane);
-    if (lane < cnt) Js[lane] = __ldg(x.crd1 + s0 + lane);
-    __syncwarp();
-
-    const int32_t N0 = Ps[0], N1 = Ps[cnt];
-    const int32_t per = (N1 - N0 + NS - 1) / NS;
-    const int32_t na = N0 + st * per;
-    const int32_t nb = na + per < N1 ? na + per : N1;
-    const bool active = na < nb;
-    int f = 0;
-    bool split = false;
-    if (active) {
-        int lo = 0, hi = cnt - 1;                                 // fibre holding node na
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (Ps[mid] <= na) lo = mid; else hi = mid - 1;
-        }
-        f = lo;
-        split = Ps[f] < na;                                       // fibre f was begun by the stream before
-    }
-    // K slot of a piece = its fibre + the number of cut fibres at or before this stream
-    const unsigned cuts = __ballot_sync(0xffffffffu, split && h == 0);
-    const int slot_off = __popc(cuts & ((2u << (st * SL)) - 1u));
-    const int nslots = cnt + __popc(cuts);
-
-    if (active) {
-        int32_t fend = Ps[f + 1];
-        float Q[2][R];
-#pragma unroll
-        for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
-
-        auto park = [&]() {                                       // rows b = 2h, 2h+1 of this piece, as they are
-            const int slot = f + slot_off;
-            float *dst = Raw + slot * RAW_ROW + 2 * h * R;
-#pragma unroll
-            for (int b2 = 0; b2 < 2; ++b2) {
-                *reinterpret_cast<float4 *>(dst + b2 * R) = make_float4(Q[b2][0], Q[b2][1], Q[b2][2], Q[b2][3]);
-                *reinterpret_cast<float4 *>(dst + b2 * R + 4) = make_float4(Q[b2][4], Q[b2][5], Q[b2][6], Q[b2][7]);
-            }
-            if (h == 0) Jslot[slot] = Js[f];
-        };
-
-        // software pipeline over the nodes of the run: descriptors two nodes ahead, rows one node ahead
-        NodeInfo cur = load_node(x, na, nb);
-        NodeInfo nxt = load_node(x, na + 1, nb);
-        float4 w0 = ldg4(W + (size_t)cur.l * R), w1 = ldg4(W + (size_t)cur.l * R + 4);
-        float2 vb = __ldg(reinterpret_cast<const float2 *>(V + (size_t)cur.k * R + 2 * h));
-        for (int32_t n = na; n < nb; ++n) {
-            const NodeInfo nn = load_node(x, n + 2, nb);
-            float4 w0n = w0, w1n = w1;
-            float2 vbn = vb;
-            if (n + 1 < nb) {
-                w0n = ldg4(W + (size_t)nxt.l * R);
-                w1n = ldg4(W + (size_t)nxt.l * R + 4);
-                vbn = __ldg(reinterpret_cast<const float2 *>(V + (size_t)nxt.k * R + 2 * h));
-            }
-            // P = sum over the node's leaves of X * W[l, :]
-            float P[R] = {cur.xv * w0.x, cur.xv * w0.y, cur.xv * w0.z, cur.xv * w0.w,
-                          cur.xv * w1.x, cur.xv * w1.y, cur.xv * w1.z, cur.xv * w1.w};
-            for (int32_t p = cur.pa + 1; p < cur.pb; ++p) {       // further leaves of the node (rare when sparse)
-                const float xv = __ldg(x.vals + p);
-                const float *w = W + (size_t)__ldg(x.crd3 + p) * R;
-                const float4 a0 = ldg4(w), a1 = ldg4(w + 4);
-                P[0] = fmaf(xv, a0.x, P[0]); P[1] = fmaf(xv, a0.y, P[1]);
-                P[2] = fmaf(xv, a0.z, P[2]); P[3] = fmaf(xv, a0.w, P[3]);
-                P[4] = fmaf(xv, a1.x, P[4]); P[5] = fmaf(xv, a1.y, P[5]);
-                P[6] = fmaf(xv, a1.z, P[6]); P[7] = fmaf(xv, a1.w, P[7]);
-            }
-#pragma unroll
-            for (int c = 0; c < R; ++c) {                         // Q[b, :] += V[k, b] * P[:]
-                Q[0][c] = fmaf(vb.x, P[c], Q[0][c]);
-                Q[1][c] = fmaf(vb.y, P[c], Q[1][c]);
-            }
-            if (n + 1 == fend) {                                  // the run leaves fibre f
-                park();
-#pragma unroll
-                for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
-                ++f;
-                fend = Ps[f + 1 <= cnt ? f + 1 : cnt];
-            }
-            cur = nxt; nxt = nn; w0 = w0n; w1 = w1n; vb = vbn;
-        }
-        if (f < cnt && nb > Ps[f]) park();                        // the run ends inside fibre f
-    }
-    __syncwarp();
-
-    // A operand: lane reads column m of four consecutive pieces (a K quad), splits, and writes 16 bytes
-    // of the hi and of the lo operand.  The pieces lie where the operands go, so the whole window is
-    // read into registers first.  Slots beyond nslots are padding and read as zero.
-    const int padded = (nslots + 7) & ~7;
-    {
-        constexpr int UNITS = SLOTS / 4 * 2;                      // (K quad, half of m) pairs per lane
-        float4 raw[UNITS];
-#pragma unroll
-        for (int u = 0; u < UNITS; ++u) {
-            const int quad = u >> 1, m = lane + 32 * (u & 1);
-            const float *src = Raw + (4 * quad) * RAW_ROW + m;
-            raw[u].x = 4 * quad + 0 < nslots ? src[0] : 0.f;
-            raw[u].y = 4 * quad + 1 < nslots ? src[RAW_ROW] : 0.f;
-            raw[u].z = 4 * quad + 2 < nslots ? src[2 * RAW_ROW] : 0.f;
-            raw[u].w = 4 * quad + 3 < nslots ? src[3 * RAW_ROW] : 0.f;
-        }
-        __syncwarp();
-#pragma unroll
-        for (int u = 0; u < UNITS; ++u) {
-            const int quad = u >> 1, m = lane + 32 * (u & 1);
-            if (4 * quad < padded) {
-                float4 hi4, lo4;
-                split4(raw[u], hi4, lo4);
-                const int off = (quad >> 1) * 512 + (quad & 1) * 256 + (m >> 3) * 32 + (m & 7) * 4;
-                *reinterpret_cast<float4 *>(Ahi + off) = hi4;
-                *reinterpret_cast<float4 *>(Alo + off) = lo4;
-            }
-        }
-    }
-    // B operand: one lane per K slot
-    const int slot = lane;
-    if (slot < padded) {
-        float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f), u1 = u0;
-        if (slot < nslots) {
-            const float *up = U + (size_t)Jslot[slot] * R;
-            u0 = ldg4(up);
-            u1 = ldg4(up + 4);
-        }
-        float4 h0, l0, h1, l1;
-        split4(u0, h0, l0);
-        split4(u1, h1, l1);
-        float *bh = Bhi + (slot >> 2) * B_QUAD + (slot & 3), *bl = Blo + (slot >> 2) * B_QUAD + (slot & 3);
-        bh[0] = h0.x; bh[4] = h0.y; bh[8] = h0.z; bh[12] = h0.w; bh[16] = h1.x; bh[20] = h1.y; bh[24] = h1.z; bh[28] = h1.w;
-        bl[0] = l0.x; bl[4] = l0.y; bl[8] = l0.z; bl[12] = l0.w; bl[16] = l1.x; bl[20] = l1.y; bl[24] = l1.z; bl[28] = l1.w;
-    }
-    return padded;
-}
-
 __global__ void __launch_bounds__(kWarps * 32)
 ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *__restrict__ light_list, Csf4 x,
                 const float *__restrict__ U, const float *__restrict__ V, const float *__restrict__ W,
@@ -337,41 +197,162 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
     float *Alo = Ahi + A_FLOATS;
     float *Bhi = Alo + A_FLOATS;
     float *Blo = Bhi + B_FLOATS;
-    int32_t *Ps = reinterpret_cast<int32_t *>(Blo + B_FLOATS);
-    int32_t *Js = Ps + 32;
-    int32_t *Jslot = Js + 32;
+    float *Raw = Blo + B_FLOATS;                                  // [SLOTS][RAW_ROW] parked pieces
+    int32_t *Jslot = reinterpret_cast<int32_t *>(Raw + SLOTS * RAW_ROW);
     const uint32_t ahi_s = smem_u32(Ahi), alo_s = smem_u32(Alo), bhi_s = smem_u32(Bhi), blo_s = smem_u32(Blo);
 
     uint32_t parity = 0;
     bool pending = false, ok = true, first = true;
-    for (int32_t s0 = fa; s0 < fb && ok; s0 += WF) {
-        const int cnt = fb - s0 < WF ? fb - s0 : WF;
-        if (pending) {                                            // the MMAs of the previous window still read the operands
+    const int st = lane / SL, h = lane % SL;
+    int cnt = 0;                                                  // pieces this stream has parked since the last flush
+
+    // Hands the parked pieces to the tensor core: Y_i += U_J^T Q_J over the 8 C slots.
+    auto flush = [&]() {
+        __syncwarp();
+        unsigned vm[C];                                           // bit s * SL of vm[c]: slot c of stream s holds a piece
+#pragma unroll
+        for (int c = 0; c < C; ++c) vm[c] = __ballot_sync(0xffffffffu, cnt > c);
+        // U rows of the slots, requested before anything waits
+        float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f), u1 = u0;
+        if (lane < SLOTS && ((vm[lane % C] >> ((lane / C) * SL)) & 1u)) {
+            const float *up = U + (size_t)Jslot[lane] * R;
+            u0 = ldg4(up);
+            u1 = ldg4(up + 4);
+        }
+        if (pending) {                                            // the MMAs of the previous flush still read the operands
             bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
             done = __shfl_sync(0xffffffffu, done, 0);
             parity ^= 1;
             pending = false;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (!done) { ok = false; break; }
+            if (!done) ok = false;
         }
-        const int padded = produce_window(x, U, V, W, s0, cnt, lane, Ahi, Alo, Bhi, Blo, Ahi, Ps, Js, Jslot);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // operand stores -> visible to the tensor core
-        __syncwarp();
-        if (lane == 0) {
-            for (int kg = 0; kg < padded / 8; ++kg) {
-                const uint64_t a_hi = smem_desc(ahi_s + kg * 2048, 1024, 128), a_lo = smem_desc(alo_s + kg * 2048, 1024, 128);
-                const uint64_t b_hi = smem_desc(bhi_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
-                const uint64_t b_lo = smem_desc(blo_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
-                umma_tf32(d_tmem, a_hi, b_hi, (first && kg == 0) ? 0u : 1u);
-                umma_tf32(d_tmem, a_lo, b_hi, 1u);
-                umma_tf32(d_tmem, a_hi, b_lo, 1u);
+        if (ok) {
+#pragma unroll
+            for (int u = 0; u < SLOTS / 2; ++u) {                 // A: (K quad, half of m) pairs
+                const int quad = u >> 1, m = lane + 32 * (u & 1);
+                float e[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int slot = 4 * quad + q;
+                    e[q] = ((vm[slot % C] >> ((slot / C) * SL)) & 1u) ? Raw[slot * RAW_ROW + m] : 0.f;
+                }
+                float4 hi4, lo4;
+                split4(make_float4(e[0], e[1], e[2], e[3]), hi4, lo4);
+                const int off = (quad >> 1) * 512 + (quad & 1) * 256 + (m >> 3) * 32 + (m & 7) * 4;
+                *reinterpret_cast<float4 *>(Ahi + off) = hi4;
+                *reinterpret_cast<float4 *>(Alo + off) = lo4;
             }
-            umma_commit(mbar);
-            acc_used[warp] = 1;
+            if (lane < SLOTS) {                                   // B: one lane per K slot
+                float4 h0, l0, h1, l1;
+                split4(u0, h0, l0);
+                split4(u1, h1, l1);
+                float *bh = Bhi + (lane >> 2) * B_QUAD + (lane & 3), *bl = Blo + (lane >> 2) * B_QUAD + (lane & 3);
+                bh[0] = h0.x; bh[4] = h0.y; bh[8] = h0.z; bh[12] = h0.w; bh[16] = h1.x; bh[20] = h1.y; bh[24] = h1.z; bh[28] = h1.w;
+                bl[0] = l0.x; bl[4] = l0.y; bl[8] = l0.z; bl[12] = l0.w; bl[16] = l1.x; bl[20] = l1.y; bl[24] = l1.z; bl[28] = l1.w;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // operand stores -> visible to the tensor core
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int kg = 0; kg < KG; ++kg) {
+                    const uint64_t a_hi = smem_desc(ahi_s + kg * 2048, 1024, 128), a_lo = smem_desc(alo_s + kg * 2048, 1024, 128);
+                    const uint64_t b_hi = smem_desc(bhi_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
+                    const uint64_t b_lo = smem_desc(blo_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
+                    umma_tf32(d_tmem, a_hi, b_hi, (first && kg == 0) ? 0u : 1u);
+                    umma_tf32(d_tmem, a_lo, b_hi, 1u);
+                    umma_tf32(d_tmem, a_hi, b_lo, 1u);
+                }
+                umma_commit(mbar);
+                acc_used[warp] = 1;
+            }
+            pending = true;
+            first = false;
         }
-        pending = true;
-        first = false;
+        cnt = 0;
         __syncwarp();
+    };
+
+    if (fa < fb) {
+        const int32_t N0 = __ldg(x.pos2 + fa), N1 = __ldg(x.pos2 + fb);
+        const int32_t per = (N1 - N0 + NS - 1) / NS;
+        const int32_t na = N0 + st * per;
+        const int32_t nb = na + per < N1 ? na + per : N1;
+        int32_t f = fa;
+        if (na < nb) {                                            // fibre holding node na
+            int32_t lo = fa, hi = fb - 1;
+            while (lo < hi) {
+                const int32_t mid = lo + (hi - lo + 1) / 2;
+                if (__ldg(x.pos2 + mid) <= na) lo = mid; else hi = mid - 1;
+            }
+            f = lo;
+        }
+        const int32_t flast = fb - 1;
+        int32_t fend = __ldg(x.pos2 + f + 1);                     // end of fibre f; the fibre after it is fetched ahead
+        int32_t fend_n = __ldg(x.pos2 + (f + 2 <= fb ? f + 2 : fb));
+        int32_t jc = __ldg(x.crd1 + f), jn = __ldg(x.crd1 + (f + 1 <= flast ? f + 1 : flast));
+        float Q[2][R];
+#pragma unroll
+        for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
+
+        // software pipeline over the nodes of the run: descriptors two nodes ahead, rows one node ahead
+        NodeInfo cur = load_node(x, na, nb);
+        NodeInfo nxt = load_node(x, na + 1, nb);
+        float4 w0 = ldg4(W + (size_t)cur.l * R), w1 = ldg4(W + (size_t)cur.l * R + 4);
+        float2 vb = __ldg(reinterpret_cast<const float2 *>(V + (size_t)cur.k * R + 2 * h));
+        for (int32_t t = 0; t < per && ok; ++t) {
+            const int32_t n = na + t;
+            const NodeInfo nn = load_node(x, n + 2, nb);
+            float4 w0n = w0, w1n = w1;
+            float2 vbn = vb;
+            if (n + 1 < nb) {
+                w0n = ldg4(W + (size_t)nxt.l * R);
+                w1n = ldg4(W + (size_t)nxt.l * R + 4);
+                vbn = __ldg(reinterpret_cast<const float2 *>(V + (size_t)nxt.k * R + 2 * h));
+            }
+            if (n < nb) {
+                // P = sum over the node's leaves of X * W[l, :]
+                float P[R] = {cur.xv * w0.x, cur.xv * w0.y, cur.xv * w0.z, cur.xv * w0.w,
+                              cur.xv * w1.x, cur.xv * w1.y, cur.xv * w1.z, cur.xv * w1.w};
+                for (int32_t p = cur.pa + 1; p < cur.pb; ++p) {   // further leaves of the node (rare when sparse)
+                    const float xv = __ldg(x.vals + p);
+                    const float *w = W + (size_t)__ldg(x.crd3 + p) * R;
+                    const float4 a0 = ldg4(w), a1 = ldg4(w + 4);
+                    P[0] = fmaf(xv, a0.x, P[0]); P[1] = fmaf(xv, a0.y, P[1]);
+                    P[2] = fmaf(xv, a0.z, P[2]); P[3] = fmaf(xv, a0.w, P[3]);
+                    P[4] = fmaf(xv, a1.x, P[4]); P[5] = fmaf(xv, a1.y, P[5]);
+                    P[6] = fmaf(xv, a1.z, P[6]); P[7] = fmaf(xv, a1.w, P[7]);
+                }
+#pragma unroll
+                for (int c = 0; c < R; ++c) {                     // Q[b, :] += V[k, b] * P[:]
+                    Q[0][c] = fmaf(vb.x, P[c], Q[0][c]);
+                    Q[1][c] = fmaf(vb.y, P[c], Q[1][c]);
+                }
+                const bool leaves = n + 1 == fend;
+                if (leaves || n + 1 == nb) {                      // the run leaves fibre f, or ends inside it: park the piece
+                    const int slot = st * C + cnt;
+                    float *dst = Raw + slot * RAW_ROW + 2 * h * R;
+#pragma unroll
+                    for (int b2 = 0; b2 < 2; ++b2) {
+                        *reinterpret_cast<float4 *>(dst + b2 * R) = make_float4(Q[b2][0], Q[b2][1], Q[b2][2], Q[b2][3]);
+                        *reinterpret_cast<float4 *>(dst + b2 * R + 4) = make_float4(Q[b2][4], Q[b2][5], Q[b2][6], Q[b2][7]);
+                        Q[b2][0] = Q[b2][1] = Q[b2][2] = Q[b2][3] = Q[b2][4] = Q[b2][5] = Q[b2][6] = Q[b2][7] = 0.f;
+                    }
+                    if (h == 0) Jslot[slot] = jc;
+                    ++cnt;
+                    if (leaves) {
+                        ++f;
+                        fend = fend_n;
+                        jc = jn;
+                        fend_n = __ldg(x.pos2 + (f + 2 <= fb ? f + 2 : fb));
+                        jn = __ldg(x.crd1 + (f + 1 <= flast ? f + 1 : flast));
+                    }
+                }
+            }
+            cur = nxt; nxt = nn; w0 = w0n; w1 = w1n; vb = vbn;
+            if (__any_sync(0xffffffffu, cnt == C)) flush();
+        }
+        if (ok && __any_sync(0xffffffffu, cnt > 0)) flush();
     }
     if (pending) {
         bool done = lane == 0 ? mbar_wait(mbar, parity) : true;

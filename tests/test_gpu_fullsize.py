@@ -74,8 +74,8 @@ def _check_csf(h, op, mode_order, rows):
         assert vals[lo:hi].cpu().numpy().tobytes() == ovals.tobytes(), f"values of slice {r}"
 
 
-@pytest.mark.parametrize("config_id", [2, 3, 4, 5])
-def test_full_size_config(config_id):
+@pytest.mark.parametrize("config_id,tensor_stage", [(2, None), (3, False), (3, True), (4, None), (5, None)])
+def test_full_size_config(config_id, tensor_stage):
     rng = np.random.default_rng(100 + config_id)
     w = make_config(config_id)
     dtype = cb.F32 if w.dtype == np.float32 else cb.F64
@@ -86,6 +86,8 @@ def test_full_size_config(config_id):
         rows_csf = _sample_rows(op, mo[0], 6, rng)
         _check_csf(handles[name], op, mo, rows_csf)
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, dtype)
+    if tensor_stage is not None:
+        cb.const_plan_set_tensor_stage(plan, tensor_stage)     # order-4 TTMc: per-slice stage on tensor cores or FMA pipes
     operands = dict(handles)
     operands.update({n: to_dev(a) for n, a in w.dense.items()})
     out = torch.full(w.out_shape, float("nan"), dtype=torch.float32 if dtype == cb.F32 else torch.float64,
