@@ -137,6 +137,8 @@ const_status_t const_plan_create(const char *expression, const char *const *tree
         delete plan;
         return rc;
     }
+    // the order-4 TTMc kernel with the per-slice stage on the tensor cores is the faster one at rank 8
+    plan->tensor_stage = plan->desc.family == Family::Ttmc4 && plan->desc.ranks[0] == 8;
     *out = plan;
     return CONST_OK;
 }
@@ -232,7 +234,7 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
 const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
     const_plan *p = const_cast<const_plan *>(as_plan(h));
     if (!p) return CONST_ERR_INVALID_ARG;
-    if (enable && p->desc.family != Family::Ttmc4) return CONST_ERR_UNSUPPORTED;
+    if (enable && !(p->desc.family == Family::Ttmc4 && p->desc.ranks[0] == 8)) return CONST_ERR_UNSUPPORTED;
     p->tensor_stage = enable ? 1 : 0;
     return CONST_OK;
 }

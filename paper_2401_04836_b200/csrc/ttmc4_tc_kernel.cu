@@ -14,6 +14,8 @@
 // fibre's j, as one piece.  The contraction is linear in Q, so a piece is simply one K slot: a fibre
 // cut between two streams occupies two slots with the same j and nothing has to be merged.  Every
 // stream owns C slots; when one of them is full the warp flushes all 8 C slots (empty ones as zeros).
+// C = 1 keeps the shared memory of a warp under 7 KB, so five blocks (twenty warps) fit on an SM, which
+// pays more than the fuller MMAs of a larger C.
 //
 // Flush.  Operands in shared memory (no swizzle, K-major, as the shared-memory matrix descriptor
 // defines it: core matrices of 8 rows x 16 bytes, i.e. 8 values of m (or n) by 4 consecutive K slots):
@@ -44,7 +46,7 @@ constexpr int R = 8;
 constexpr int TILE = R * R * R;   // floats of one output row (slice)
 constexpr int SL = 4;             // lanes per node stream
 constexpr int NS = 32 / SL;       // node streams per warp
-constexpr int C = 2;              // K slots (parked pieces) per stream between two flushes
+constexpr int C = 1;              // K slots (parked pieces) per stream between two flushes
 constexpr int SLOTS = NS * C;     // K slots per flush
 constexpr int KG = SLOTS / 8;     // groups of eight slots = MMAs per operand pair
 constexpr int kWarps = 4;
@@ -137,7 +139,7 @@ __device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t 
     return r;
 }
 
-__global__ void __launch_bounds__(kWarps * 32)
+__global__ void __launch_bounds__(kWarps * 32, 5)
 ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *__restrict__ light_list, Csf4 x,
                 const float *__restrict__ U, const float *__restrict__ V, const float *__restrict__ W,
                 float *__restrict__ out, int32_t *__restrict__ status) {

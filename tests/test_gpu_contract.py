@@ -75,29 +75,21 @@ def test_mttkrp_each_bin(rank, bins):
     check(w, bins)
 
 
+# order-4 TTMc: the per-slice stage Y_i = U_J^T Q_J runs on the tensor cores (split tf32 operands, the
+# default at rank 8) or on the FMA pipes; both must meet the fp32 tolerance
+@pytest.mark.parametrize("tensor_stage", [False, True])
 @pytest.mark.parametrize("bins", [None, ALL_LIGHT, ALL_HEAVY, ALL_GIANT, MIXED])
-def test_ttmc4_each_bin(bins):
+def test_ttmc4_each_bin(bins, tensor_stage):
     w = ttmc4_workload((300, 40, 30, 50), 80_000, 8, slice_s=1.0, value="pm1", config_id=3)
-    check(w, bins)
+    check(w, bins, tensor_stage=tensor_stage)
 
 
-def test_ttmc4_sparse_like_the_benchmark():
+@pytest.mark.parametrize("tensor_stage", [False, True, None])
+def test_ttmc4_sparse_like_the_benchmark(tensor_stage):
     w = make_config(3, scale=0.004)             # 200k nonzeros in 20000^4: every (i,j,k) fibre has one leaf
-    check(w)
-
-
-@pytest.mark.parametrize("bins", [None, ALL_LIGHT, ALL_HEAVY, ALL_GIANT, MIXED])
-def test_ttmc4_tensor_stage_each_bin(bins):
-    # the per-slice stage Y_i = U_J^T Q_J on the tensor cores (split tf32 operands) meets the fp32 tolerance
-    w = ttmc4_workload((300, 40, 30, 50), 80_000, 8, slice_s=1.0, value="pm1", config_id=3)
-    check(w, bins, tensor_stage=True)
-
-
-def test_ttmc4_tensor_stage_sparse_like_the_benchmark():
-    w = make_config(3, scale=0.004)
-    check(w, tensor_stage=True)
+    check(w, tensor_stage=tensor_stage)
     w = ttmc4_workload((7, 5, 3, 4), 60, 8, slice_s=1.0, value="pm1", config_id=3)      # a handful of tiny slices
-    check(w, tensor_stage=True)
+    check(w, tensor_stage=tensor_stage)
 
 
 def test_tensor_stage_only_where_a_kernel_has_one():
