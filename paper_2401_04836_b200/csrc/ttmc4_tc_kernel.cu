@@ -32,9 +32,10 @@
 // memory; the dropped lo*lo term and the truncation of lo are below 2^-20 relative per term.
 //
 // A block has four warps because a warp can read only its own quarter of the 128 tensor-memory
-// lanes (rows 16w..16w+15 of an M = 64 accumulator live in lanes 32w..32w+15).  Work items are
-// sized for kWarpsPerBlock warps, so a block takes kWarps / kWarpsPerBlock consecutive items; every
-// warp owns an 8-column accumulator and the epilogue adds the accumulators of an item's warps.
+// lanes (rows 16w..16w+15 of an M = 64 accumulator live in lanes 32w..32w+15).  A block takes one
+// work item: the four warps cut the fibres of a heavy slice or chunk in four by leaf count, and a
+// light item (up to kWarpsPerBlock slices) gives each slice to kWarps / kWarpsPerBlock warps.  Every
+// warp owns an 8-column accumulator and the epilogue adds the accumulators that belong to one slice.
 // Every wait on an mbarrier is bounded; on a timeout the block records CONST_ERR_TIMEOUT in the
 // status word, stops issuing MMAs, skips its stores and still frees its tensor memory.
 #include "common.cuh"
@@ -50,7 +51,7 @@ constexpr int C = 1;              // K slots (parked pieces) per stream between 
 constexpr int SLOTS = NS * C;     // K slots per flush
 constexpr int KG = SLOTS / 8;     // groups of eight slots = MMAs per operand pair
 constexpr int kWarps = 4;
-constexpr int kItemsPerBlock = kWarps / kWarpsPerBlock;
+constexpr int kWarpsPerLight = kWarps / kWarpsPerBlock;    // warps per slice of a light item
 constexpr int kTmemCols = 32;     // kWarps accumulators of 8 columns
 static_assert(SLOTS % 8 == 0 && SLOTS <= 32, "one lane per slot when the B operand is written");
 
@@ -148,30 +149,30 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
     __shared__ uint32_t tmem_base_s;
     __shared__ int32_t acc_row[kWarps];          // output row of every warp's accumulator, -1: none
     __shared__ int32_t acc_used[kWarps];         // the warp issued at least one MMA
-    __shared__ int32_t item_kind[kItemsPerBlock];
     __shared__ int32_t failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int item_slot = warp / kWarpsPerBlock, wl = warp % kWarpsPerBlock;
-    const int64_t item_idx = (int64_t)blockIdx.x * kItemsPerBlock + item_slot;
-    const bool have = item_idx < n_items;
-    WorkItem it{0, 0, 0, kItemLight};
-    if (have) it = items[item_idx];
+    const WorkItem it = items[blockIdx.x];
     const bool light = it.kind == kItemLight;
 
-    int32_t slice = it.slice, fa = 0, fb = 0;
+    // this warp's share: part `part` of `parts` of the level-1 nodes [f0, f1) of `slice`, cut by leaf count
+    int32_t slice = it.slice, f0 = it.f0, f1 = it.f1, fa = 0, fb = 0;
+    int part = warp, parts = kWarps;
     if (light) {
-        if (wl < it.f0) {
-            slice = __ldg(light_list + it.slice + wl);
-            fa = __ldg(x.pos1 + slice);
-            fb = __ldg(x.pos1 + slice + 1);
+        const int sl = warp / kWarpsPerLight;
+        part = warp % kWarpsPerLight;
+        parts = kWarpsPerLight;
+        f0 = f1 = 0;
+        if (sl < it.f0) {
+            slice = __ldg(light_list + it.slice + sl);
+            f0 = __ldg(x.pos1 + slice);
+            f1 = __ldg(x.pos1 + slice + 1);
         }
-    } else {
-        const int64_t lo = leaf_of(x, it.f0), hi = leaf_of(x, it.f1);
-        fa = wl == 0 ? it.f0 : lower_bound_leaf(x, it.f0, it.f1, lo + (hi - lo) * wl / kWarpsPerBlock);
-        fb = wl == kWarpsPerBlock - 1
-                 ? it.f1
-                 : lower_bound_leaf(x, it.f0, it.f1, lo + (hi - lo) * (wl + 1) / kWarpsPerBlock);
+    }
+    if (f0 < f1) {
+        const int64_t lo = leaf_of(x, f0), hi = leaf_of(x, f1);
+        fa = part == 0 ? f0 : lower_bound_leaf(x, f0, f1, lo + (hi - lo) * part / parts);
+        fb = part == parts - 1 ? f1 : lower_bound_leaf(x, f0, f1, lo + (hi - lo) * (part + 1) / parts);
     }
 
     const uint32_t mbar = smem_u32(&mbar_all[warp]);
@@ -179,7 +180,6 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar) : "memory");
         acc_row[warp] = fa < fb ? __ldg(x.crd0 + slice) : -1;
         acc_used[warp] = 0;
-        if (wl == 0) item_kind[item_slot] = it.kind;
         if (warp == 0) failed = 0;
     }
     __syncwarp();
@@ -383,42 +383,32 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (lane < 16) {
             const int m = 16 * warp + lane;
+            // accumulators of the same slice are added: all four for a heavy slice or chunk,
+            // kWarpsPerLight neighbours for every slice of a light item
+            const int group = light ? kWarpsPerLight : kWarps;
 #pragma unroll
-            for (int p = 0; p < kItemsPerBlock; ++p) {
-                const int kind = item_kind[p];
-                if (kind == kItemLight) {
+            for (int g0 = 0; g0 < kWarps; g0 += kWarpsPerLight) {
+                if (g0 % group != 0) continue;
+                float sum[R];
+                int row = -1;
 #pragma unroll
-                    for (int q = 0; q < kWarpsPerBlock; ++q) {
-                        const int a = p * kWarpsPerBlock + q;
-                        if (acc_row[a] >= 0 && acc_used[a]) {
-                            float *dst = out + (size_t)acc_row[a] * TILE + m;
+                for (int n = 0; n < R; ++n) sum[n] = 0.f;
 #pragma unroll
-                            for (int n = 0; n < R; ++n) dst[n * 64] = __uint_as_float(r[a][n]);
-                        }
+                for (int a = 0; a < kWarps; ++a) {
+                    if (a >= g0 && a < g0 + group && acc_row[a] >= 0 && acc_used[a]) {
+                        row = acc_row[a];
+#pragma unroll
+                        for (int n = 0; n < R; ++n) sum[n] += __uint_as_float(r[a][n]);
                     }
-                } else {
-                    float sum[R];
-                    int row = -1;
+                }
+                if (row >= 0) {
+                    float *dst = out + (size_t)row * TILE + m;
+                    if (it.kind == kItemChunk) {
 #pragma unroll
-                    for (int n = 0; n < R; ++n) sum[n] = 0.f;
+                        for (int n = 0; n < R; ++n) atomicAdd(dst + n * 64, sum[n]);
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < kWarpsPerBlock; ++q) {
-                        const int a = p * kWarpsPerBlock + q;
-                        if (acc_row[a] >= 0 && acc_used[a]) {
-                            row = acc_row[a];
-#pragma unroll
-                            for (int n = 0; n < R; ++n) sum[n] += __uint_as_float(r[a][n]);
-                        }
-                    }
-                    if (row >= 0) {
-                        float *dst = out + (size_t)row * TILE + m;
-                        if (kind == kItemBlock) {
-#pragma unroll
-                            for (int n = 0; n < R; ++n) dst[n * 64] = sum[n];
-                        } else {
-#pragma unroll
-                            for (int n = 0; n < R; ++n) atomicAdd(dst + n * 64, sum[n]);
-                        }
+                        for (int n = 0; n < R; ++n) dst[n * 64] = sum[n];
                     }
                 }
             }
@@ -447,7 +437,7 @@ const_status_t run_ttmc4_tensor(const const_csf *X, const float *U, const float 
         CB_CUDA(cudaFuncSetAttribute(ttmc4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const unsigned grid = (unsigned)((X->n_items + kItemsPerBlock - 1) / kItemsPerBlock);
+    const unsigned grid = (unsigned)X->n_items;
     CB_LAUNCH("ttmc4_tc_kernel", stream,
               ttmc4_tc_kernel<<<grid, kWarps * 32, dyn, stream>>>(X->items, (int)X->n_items, X->light_list, x, U, V, W, Y, status));
     CB_CUDA(cudaGetLastError());
