@@ -181,6 +181,7 @@ def main():
     ap.add_argument("--oracle-nnz", type=int, default=0, help="nonzeros in the CPU-baseline sample (0 = auto)")
     ap.add_argument("--tensor-stage", type=int, default=-1,
                     help="order-4 TTMc: 1 = dense per-slice stage on the tensor cores, 0 = on the FMA pipes, -1 = library default")
+    ap.add_argument("--bins", default="", help="light_max,heavy_max,chunk nonzero thresholds of the load balancer (default: the library's)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernels)")
     args = ap.parse_args()
@@ -248,8 +249,17 @@ def main():
         cb.const_plan_set_tensor_stage(plan, bool(args.tensor_stage))
     stream = torch.cuda.current_stream()
 
+    bins_override = tuple(int(x) for x in args.bins.split(",")) if args.bins else None
+
+    def build_all(src):
+        hs = {n: cb.const_csf_build(cs, v, w.sparse[n].dims, w.mode_orders[n]) for n, (cs, v) in src.items()}
+        if bins_override:
+            for h in hs.values():
+                cb.const_csf_set_bins(h, *bins_override)
+        return hs
+
     def step(src, dense):
-        handles = {n: cb.const_csf_build(cs, v, w.sparse[n].dims, w.mode_orders[n]) for n, (cs, v) in src.items()}
+        handles = build_all(src)
         ops = dict(handles)
         ops.update(dense)
         cb.const_execute(plan, ops, out)
@@ -296,7 +306,7 @@ def main():
     mids = []
     for s in range(args.steps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        handles = {n: cb.const_csf_build(cs, v, w.sparse[n].dims, w.mode_orders[n]) for n, (cs, v) in dev.items()}
+        handles = build_all(dev)
         a.record(stream)
         ops = dict(handles); ops.update(dev_dense)
         cb.const_execute(plan, ops, out)

@@ -13,7 +13,8 @@
 // registers.  When a stream's run leaves a fibre, or ends, its lanes park their part of Q, with the
 // fibre's j, as one piece.  The contraction is linear in Q, so a piece is simply one K slot: a fibre
 // cut between two streams occupies two slots with the same j and nothing has to be merged.  Every
-// stream owns C slots; when one of them is full the warp flushes all 8 C slots (empty ones as zeros).
+// stream owns C slots; when a stream has to park and finds them taken, the warp flushes all 8 C slots
+// (empty ones as zeros).
 // C = 1 keeps the shared memory of a warp under 7 KB, so five blocks (twenty warps) fit on an SM, which
 // pays more than the fuller MMAs of a larger C.
 //
@@ -312,6 +313,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
                 w1n = ldg4(W + (size_t)nxt.l * R + 4);
                 vbn = __ldg(reinterpret_cast<const float2 *>(V + (size_t)nxt.k * R + 2 * h));
             }
+            bool parks = false;
             if (n < nb) {
                 // P = sum over the node's leaves of X * W[l, :]
                 float P[R] = {cur.xv * w0.x, cur.xv * w0.y, cur.xv * w0.z, cur.xv * w0.w,
@@ -330,29 +332,30 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
                     Q[0][c] = fmaf(vb.x, P[c], Q[0][c]);
                     Q[1][c] = fmaf(vb.y, P[c], Q[1][c]);
                 }
-                const bool leaves = n + 1 == fend;
-                if (leaves || n + 1 == nb) {                      // the run leaves fibre f, or ends inside it: park the piece
-                    const int slot = st * C + cnt;
-                    float *dst = Raw + slot * RAW_ROW + 2 * h * R;
+                parks = n + 1 == fend || n + 1 == nb;             // the run leaves fibre f, or ends inside it
+            }
+            // flush as late as possible: only when a stream that has to park finds its slots taken
+            if (__any_sync(0xffffffffu, parks && cnt == C)) flush();
+            if (parks && ok) {
+                const int slot = st * C + cnt;
+                float *dst = Raw + slot * RAW_ROW + 2 * h * R;
 #pragma unroll
-                    for (int b2 = 0; b2 < 2; ++b2) {
-                        *reinterpret_cast<float4 *>(dst + b2 * R) = make_float4(Q[b2][0], Q[b2][1], Q[b2][2], Q[b2][3]);
-                        *reinterpret_cast<float4 *>(dst + b2 * R + 4) = make_float4(Q[b2][4], Q[b2][5], Q[b2][6], Q[b2][7]);
-                        Q[b2][0] = Q[b2][1] = Q[b2][2] = Q[b2][3] = Q[b2][4] = Q[b2][5] = Q[b2][6] = Q[b2][7] = 0.f;
-                    }
-                    if (h == 0) Jslot[slot] = jc;
-                    ++cnt;
-                    if (leaves) {
-                        ++f;
-                        fend = fend_n;
-                        jc = jn;
-                        fend_n = __ldg(x.pos2 + (f + 2 <= fb ? f + 2 : fb));
-                        jn = __ldg(x.crd1 + (f + 1 <= flast ? f + 1 : flast));
-                    }
+                for (int b2 = 0; b2 < 2; ++b2) {
+                    *reinterpret_cast<float4 *>(dst + b2 * R) = make_float4(Q[b2][0], Q[b2][1], Q[b2][2], Q[b2][3]);
+                    *reinterpret_cast<float4 *>(dst + b2 * R + 4) = make_float4(Q[b2][4], Q[b2][5], Q[b2][6], Q[b2][7]);
+                    Q[b2][0] = Q[b2][1] = Q[b2][2] = Q[b2][3] = Q[b2][4] = Q[b2][5] = Q[b2][6] = Q[b2][7] = 0.f;
+                }
+                if (h == 0) Jslot[slot] = jc;
+                ++cnt;
+                if (n + 1 == fend) {
+                    ++f;
+                    fend = fend_n;
+                    jc = jn;
+                    fend_n = __ldg(x.pos2 + (f + 2 <= fb ? f + 2 : fb));
+                    jn = __ldg(x.crd1 + (f + 1 <= flast ? f + 1 : flast));
                 }
             }
             cur = nxt; nxt = nn; w0 = w0n; w1 = w1n; vb = vbn;
-            if (__any_sync(0xffffffffu, cnt == C)) flush();
         }
         if (ok && __any_sync(0xffffffffu, cnt > 0)) flush();
     }
