@@ -129,14 +129,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
 
 struct NodeInfo { int32_t k, pa, pb, l; float xv; };      // one level-2 node and its first leaf
 
-__device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t n_end) {
-    NodeInfo r{0, 0, 0, 0, 0.f};
+// `pa` is the node's first leaf: the end of the node before it, which the caller already holds, so no
+// address here waits for a load of the same call.
+__device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t n_end, int32_t pa) {
+    NodeInfo r{0, pa, pa, 0, 0.f};
     if (n < n_end) {
         r.k = __ldg(x.crd2 + n);
-        r.pa = __ldg(x.pos3 + n);
         r.pb = __ldg(x.pos3 + n + 1);
-        r.l = __ldg(x.crd3 + r.pa);
-        r.xv = __ldg(x.vals + r.pa);
+        r.l = __ldg(x.crd3 + pa);
+        r.xv = __ldg(x.vals + pa);
     }
     return r;
 }
@@ -299,13 +300,13 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
         for (int c = 0; c < R; ++c) Q[0][c] = Q[1][c] = 0.f;
 
         // software pipeline over the nodes of the run: descriptors two nodes ahead, rows one node ahead
-        NodeInfo cur = load_node(x, na, nb);
-        NodeInfo nxt = load_node(x, na + 1, nb);
+        NodeInfo cur = load_node(x, na, nb, na < nb ? __ldg(x.pos3 + na) : 0);
+        NodeInfo nxt = load_node(x, na + 1, nb, cur.pb);
         float4 w0 = ldg4(W + (size_t)cur.l * R), w1 = ldg4(W + (size_t)cur.l * R + 4);
         float2 vb = __ldg(reinterpret_cast<const float2 *>(V + (size_t)cur.k * R + 2 * h));
         for (int32_t t = 0; t < per && ok; ++t) {
             const int32_t n = na + t;
-            const NodeInfo nn = load_node(x, n + 2, nb);
+            const NodeInfo nn = load_node(x, n + 2, nb, nxt.pb);
             float4 w0n = w0, w1n = w1;
             float2 vbn = vb;
             if (n + 1 < nb) {
