@@ -33,9 +33,10 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FMA lanes
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 
 # DRAM bytes per nonzero and launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of
-# config 2 at scale 0.3 summarised under profiles/; both kernels stream their inputs once, so the traffic
+# configs 2 and 3 at scale 0.3 summarised under profiles/; the kernels stream their inputs once, so the traffic
 # of a full-size launch is this figure times its nonzero count.  Only valid for that workload family.
-NCU_TRAFFIC_BYTES_PER_NNZ = {("ttmc3", "rs_onesweep"): 526.0e6 / 23.1e6, ("ttmc3", "chain3_kernel"): 236.6e6 / 23.1e6}
+NCU_TRAFFIC_BYTES_PER_NNZ = {("ttmc3", "rs_onesweep"): 530.7e6 / 23.1e6, ("ttmc3", "chain3_kernel"): 235.8e6 / 23.1e6,
+                             ("ttmc4", "ttmc4_tc_kernel"): 352.9e6 / 15.0e6}
 
 
 def measured_peaks():
