@@ -68,6 +68,41 @@ def test_ttmc3_other_mode_at_the_root():
     assert_close(out.cpu().numpy(), S, A, np.float32)
 
 
+@pytest.mark.parametrize("root", [0, 1, 2])
+@pytest.mark.parametrize("family", ["mttkrp", "ttmc"])
+def test_every_output_mode(family, root):
+    """All three MTTKRPs (Sec. 5.2) and TTMcs (Sec. 5.3) of one tensor: the output is indexed by mode `root`,
+    so the schedule stores the tensor with that mode at the CSF root and contracts the other two."""
+    from oracle import contract as oc
+    dims, rank = (70, 55, 45), 16
+    w = ttmc3_workload(dims, 8_000, rank, slice_s=1.0, inner_s=None, value="pm1", config_id=11)
+    X = w.sparse["X"]
+    p, q = [m for m in range(3) if m != root]
+    names = "ijk"
+    r_, p_, q_ = names[root], names[p], names[q]
+    rng = np.random.default_rng(5)
+    Fp = rng.standard_normal((dims[p], rank)).astype(np.float32)
+    Fq = rng.standard_normal((dims[q], rank)).astype(np.float32)
+    ext = {"i": dims[0], "j": dims[1], "k": dims[2], "x": rank, "z": rank}
+    h = build_csf(X, (root, p, q))
+    coords = [X.coords[root], X.coords[p], X.coords[q]]
+    if family == "mttkrp":
+        plan = cb.const_plan_create(f"O[{r_},z] = X[i,j,k] * P[{p_},z] * Q[{q_},z]",
+                                    [f"T[{r_},{p_},z] = X[i,j,k] * Q[{q_},z]", f"O[{r_},z] = T[{r_},{p_},z] * P[{p_},z]"],
+                                    {"X": (root, p, q)}, [f"{r_}{p_}{q_}z", f"{r_}{p_}z"], ext, cb.F32)
+        out = torch.full((dims[root], rank), float("nan"), device="cuda")
+        S, A = oc.mttkrp3(coords, X.vals, Fp, Fq, dims[root])
+    else:
+        plan = cb.const_plan_create(f"O[{r_},x,z] = X[i,j,k] * P[{p_},x] * Q[{q_},z]",
+                                    [f"T[{r_},{p_},z] = X[i,j,k] * Q[{q_},z]", f"O[{r_},x,z] = T[{r_},{p_},z] * P[{p_},x]"],
+                                    {"X": (root, p, q)}, [f"{r_}{p_}{q_}z", f"{r_}{p_}xz"], ext, cb.F32)
+        out = torch.full((dims[root], rank, rank), float("nan"), device="cuda")
+        S, A = oc.ttmc3(coords, X.vals, Fp, Fq, dims[root])
+    cb.const_execute(plan, {"X": h, "P": to_dev(Fp), "Q": to_dev(Fq)}, out)
+    assert cb.const_last_device_status(plan) == 0
+    assert_close(out.cpu().numpy(), S, A, np.float32)
+
+
 @pytest.mark.parametrize("bins", [None, ALL_LIGHT, ALL_GIANT, MIXED])
 @pytest.mark.parametrize("rank", [8, 16, 32])
 def test_mttkrp_each_bin(rank, bins):
