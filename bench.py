@@ -181,7 +181,7 @@ def main():
     ap.add_argument("--impl", default="const")
     ap.add_argument("--oracle-nnz", type=int, default=0, help="nonzeros in the CPU-baseline sample (0 = auto)")
     ap.add_argument("--tensor-stage", type=int, default=-1,
-                    help="order-4 TTMc: 1 = dense per-slice stage on the tensor cores, 0 = on the FMA pipes, -1 = library default")
+                    help="TTMc: 1 = dense per-slice stage on the tensor cores, 0 = on the FMA pipes, -1 = library default")
     ap.add_argument("--bins", default="", help="light_max,heavy_max,chunk nonzero thresholds of the load balancer (default: the library's)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernels)")
@@ -246,7 +246,7 @@ def main():
     out = torch.empty(w.out_shape, dtype=tdtype, device="cuda")
     out_host = torch.empty(w.out_shape, dtype=tdtype).pin_memory()
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, dtype)
-    if args.tensor_stage >= 0 and w.family == "ttmc4":
+    if args.tensor_stage >= 0 and w.family in ("ttmc4", "ttmc3"):
         cb.const_plan_set_tensor_stage(plan, bool(args.tensor_stage))
     stream = torch.cuda.current_stream()
 
@@ -361,7 +361,7 @@ def main():
     kernels = [{"name": k, "launches": n, "ms_total": round(ms, 4), "share": round(ms / ksum, 4)}
                for k, (n, ms) in sorted(prof.items(), key=lambda kv: -kv[1][1])]
     gpu_launches = int(sum(n for n, _ in prof.values()))
-    fused_names = {"chain3_kernel", "ttmc4_kernel", "ttmc4_tc_kernel", "network_kernel"}
+    fused_names = {"chain3_kernel", "chain3_tc_kernel", "ttmc4_kernel", "ttmc4_tc_kernel", "network_kernel"}
     vbytes = w.dtype.itemsize
 
     def traffic_of(name):

@@ -203,6 +203,9 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
     const int64_t n_rows = d.extents.at(d.result.idx[0]);
     switch (d.family) {
         case Family::Ttmc3:
+            if (p->tensor_stage)
+                return run_ttmc3_tensor(X, (const float *)dense[0], (const float *)dense[1], d.ranks[0], d.ranks[1],
+                                        (float *)out_dev, n_rows, p->status_dev, stream);
             return run_ttmc3(X, (const float *)dense[0], (const float *)dense[1], d.ranks[0], d.ranks[1],
                              (float *)out_dev, n_rows, p->status_dev, stream);
         case Family::Mttkrp3:
@@ -234,7 +237,9 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
 const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
     const_plan *p = const_cast<const_plan *>(as_plan(h));
     if (!p) return CONST_ERR_INVALID_ARG;
-    if (enable && !(p->desc.family == Family::Ttmc4 && p->desc.ranks[0] == 8)) return CONST_ERR_UNSUPPORTED;
+    const bool has_stage = (p->desc.family == Family::Ttmc4 && p->desc.ranks[0] == 8) ||
+                           (p->desc.family == Family::Ttmc3 && p->desc.ranks[0] == 16 && p->desc.ranks[1] == 16);
+    if (enable && !has_stage) return CONST_ERR_UNSUPPORTED;
     p->tensor_stage = enable ? 1 : 0;
     return CONST_OK;
 }

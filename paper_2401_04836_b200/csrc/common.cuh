@@ -107,6 +107,9 @@ const_status_t run_ttmc4(const const_csf *X, const float *U, const float *V, con
 // ttmc4_tc_kernel.cu: the same contraction with the per-slice dense stage on the tensor cores
 const_status_t run_ttmc4_tensor(const const_csf *X, const float *U, const float *V, const float *W, int R, float *Y,
                                 int64_t n_rows, int32_t *status, cudaStream_t stream);
+// chain3_tc_kernel.cu: order-3 TTMc at rank 16 x 16 with the per-slice dense stage on the tensor cores
+const_status_t run_ttmc3_tensor(const const_csf *X, const float *U, const float *V, int R2, int R3, float *Y,
+                                int64_t n_rows, int32_t *status, cudaStream_t stream);
 // network_kernels.cu
 const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z,
                            int64_t n_i, int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m,

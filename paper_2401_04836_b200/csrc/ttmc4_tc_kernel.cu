@@ -40,9 +40,12 @@
 // Every wait on an mbarrier is bounded; on a timeout the block records CONST_ERR_TIMEOUT in the
 // status word, stops issuing MMAs, skips its stores and still frees its tensor memory.
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace cb {
 namespace {
+
+using namespace umma;
 
 constexpr int R = 8;
 constexpr int TILE = R * R * R;   // floats of one output row (slice)
@@ -65,14 +68,12 @@ constexpr int WARP_INTS = 32;             // Jslot[SLOTS]
 constexpr size_t kWarpBytes = (sizeof(float) * WARP_FLOATS + sizeof(int32_t) * WARP_INTS + 127) / 128 * 128;
 
 // instruction descriptor: D fp32, A and B tf32, both K-major, N = 8, M = 64
-constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((8u >> 3) << 17) | ((64u >> 4) << 24);
+constexpr uint32_t kIdesc = idesc_tf32(64, 8);
 
 struct Csf4 {
     const int32_t *crd0, *pos1, *crd1, *pos2, *crd2, *pos3, *crd3;
     const float *vals;
 };
-
-__device__ __forceinline__ float4 ldg4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 
 __device__ __forceinline__ int32_t leaf_of(const Csf4 &x, int32_t f1) { return __ldg(x.pos3 + __ldg(x.pos2 + f1)); }
 
@@ -82,49 +83,6 @@ __device__ __forceinline__ int32_t lower_bound_leaf(const Csf4 &x, int32_t lo, i
         if ((int64_t)leaf_of(x, mid) < target) lo = mid + 1; else hi = mid;
     }
     return lo;
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ float tf32_rn(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
-}
-
-__device__ __forceinline__ void split4(const float4 &x, float4 &hi, float4 &lo) {
-    hi = make_float4(tf32_rn(x.x), tf32_rn(x.y), tf32_rn(x.z), tf32_rn(x.w));
-    lo = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
-}
-
-// shared-memory matrix descriptor, no swizzle: start address, K-direction ("leading") and
-// MN-direction ("stride") byte offsets between core matrices, all in 16-byte units
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-           (1ull << 46);
-}
-
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint32_t mbar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(mbar) : "memory");
-}
-
-// true when the phase with the given parity has completed; gives up after a bounded number of polls
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
-    for (int it = 0; it < (1 << 20); ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
-        if (ok) return true;
-    }
-    return false;
 }
 
 struct NodeInfo { int32_t k, pa, pb, l; float xv; };      // one level-2 node and its first leaf
@@ -263,9 +221,9 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
                     const uint64_t a_hi = smem_desc(ahi_s + kg * 2048, 1024, 128), a_lo = smem_desc(alo_s + kg * 2048, 1024, 128);
                     const uint64_t b_hi = smem_desc(bhi_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
                     const uint64_t b_lo = smem_desc(blo_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
-                    umma_tf32(d_tmem, a_hi, b_hi, (first && kg == 0) ? 0u : 1u);
-                    umma_tf32(d_tmem, a_lo, b_hi, 1u);
-                    umma_tf32(d_tmem, a_hi, b_lo, 1u);
+                    umma_tf32(d_tmem, a_hi, b_hi, kIdesc, (first && kg == 0) ? 0u : 1u);
+                    umma_tf32(d_tmem, a_lo, b_hi, kIdesc, 1u);
+                    umma_tf32(d_tmem, a_hi, b_lo, kIdesc, 1u);
                 }
                 umma_commit(mbar);
                 acc_used[warp] = 1;

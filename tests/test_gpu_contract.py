@@ -127,6 +127,22 @@ def test_ttmc4_sparse_like_the_benchmark(tensor_stage):
     check(w, tensor_stage=tensor_stage)
 
 
+@pytest.mark.parametrize("tensor_stage", [False, True])
+@pytest.mark.parametrize("bins", [None, ALL_LIGHT, ALL_HEAVY, ALL_GIANT, MIXED])
+def test_ttmc3_rank16_tensor_stage_each_bin(bins, tensor_stage):
+    # order-3 TTMc at rank 16 x 16: Y_i = T_J^T U_J on the tensor cores (split tf32 operands) or on the FMA pipes
+    w = ttmc3_workload((500, 300, 700), 120_000, 16, slice_s=1.1, inner_s=0.9, value="unit", config_id=2)
+    check(w, bins, tensor_stage=tensor_stage)
+    w = ttmc3_workload((40, 30, 5000), 150_000, 16, slice_s=1.0, inner_s=None, value="pm1", config_id=7)   # long fibres
+    check(w, bins, tensor_stage=tensor_stage)
+
+
+def test_ttmc3_rank16_tensor_stage_tiny():
+    w = ttmc3_workload((7, 5, 6), 40, 16, value="pm1", config_id=12)
+    check(w, tensor_stage=True)
+    check(make_config(2, scale=0.005), tensor_stage=True)
+
+
 def test_tensor_stage_only_where_a_kernel_has_one():
     w = make_config(1)
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, cb.F32)
