@@ -196,13 +196,14 @@ const_status_t const_execute(const_plan_t *plan, const const_operand_t *operands
                              void *out_dev, void *stream);
 
 /*
- * Choose where the dense per-slice stage of a plan runs.  The last contraction of an order-4 TTMc,
- * summed over the fibres of a slice, is the contraction Y_i = U_J^T * Q_J (K = fibres of the slice;
- * the consumer statement of the Fig. 4(b) structure regrouped).  enable != 0: const_execute runs it
- * on the tensor cores (tcgen05, tf32 operands split into two terms each, fp32 accumulation in
- * tensor memory: per-term relative error below 2^-19, so the fp32 tolerance holds); enable == 0:
- * on the fp32 FMA pipes.  Only plans of the order-4 TTMc family with rank 8 have the stage, and for
- * them const_plan_create switches it on; CONST_ERR_UNSUPPORTED for enable != 0 on any other plan.  Host-only call; takes effect at the next
+ * Choose where the dense per-slice stage of a plan runs.  The last contraction of a TTMc, summed over
+ * the fibres of a slice, is the contraction Y_i = U_J^T * T_J (K = fibres of the slice; the consumer
+ * statement of the Fig. 4(b) structure regrouped).  enable != 0: const_execute runs it on the tensor
+ * cores (tcgen05, tf32 operands split into two terms each, fp32 accumulation in tensor memory:
+ * per-term relative error below 2^-19, so the fp32 tolerance holds); enable == 0: on the fp32 FMA pipes.
+ * Plans that have the stage: order-4 TTMc at rank 8 (const_plan_create switches it on: it is the faster
+ * path) and order-3 TTMc at rank 16 x 16 (off unless asked for: the FMA path is faster there).
+ * CONST_ERR_UNSUPPORTED for enable != 0 on any other plan.  Host-only call; takes effect at the next
  * const_execute.  A device-side wait that runs out is reported through const_last_device_status.
  */
 const_status_t const_plan_set_tensor_stage(const_plan_t *plan, int enable);

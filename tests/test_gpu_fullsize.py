@@ -74,7 +74,7 @@ def _check_csf(h, op, mode_order, rows):
         assert vals[lo:hi].cpu().numpy().tobytes() == ovals.tobytes(), f"values of slice {r}"
 
 
-@pytest.mark.parametrize("config_id,tensor_stage", [(2, None), (3, False), (3, True), (4, None), (5, None)])
+@pytest.mark.parametrize("config_id,tensor_stage", [(2, None), (2, True), (3, False), (3, True), (4, None), (5, None)])
 def test_full_size_config(config_id, tensor_stage):
     rng = np.random.default_rng(100 + config_id)
     w = make_config(config_id)
@@ -87,7 +87,7 @@ def test_full_size_config(config_id, tensor_stage):
         _check_csf(handles[name], op, mo, rows_csf)
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, dtype)
     if tensor_stage is not None:
-        cb.const_plan_set_tensor_stage(plan, tensor_stage)     # order-4 TTMc: per-slice stage on tensor cores or FMA pipes
+        cb.const_plan_set_tensor_stage(plan, tensor_stage)     # TTMc: per-slice stage on tensor cores or FMA pipes
     operands = dict(handles)
     operands.update({n: to_dev(a) for n, a in w.dense.items()})
     out = torch.full(w.out_shape, float("nan"), dtype=torch.float32 if dtype == cb.F32 else torch.float64,
