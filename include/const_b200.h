@@ -196,6 +196,24 @@ const_status_t const_execute(const_plan_t *plan, const const_operand_t *operands
                              void *out_dev, void *stream);
 
 /*
+ * Concrete index notation of a schedule (Sec. 4.2, Algorithm 1 `generate` with its helper `remove`):
+ * the contractions, each with its loop permutation, become a nest of forall(index, ...) and
+ * where(consumer, producer) constructs, e.g. for the running example of Sec. 4.1
+ *   forall(r, forall(j, where(forall(k, forall(i, R(j, k, i) = Y(k, i) * D(r, j, k))), where(...))))
+ * References are printed in stored order (a CSF input by its mode order, an intermediate by the loop
+ * order of its producer) and an intermediate loses every index whose forall encloses both its
+ * producer and its consumer.  Arguments as for const_plan_create; validate != 0 runs the Sec. 3.2
+ * checks first (CONST_ERR_ILLEGAL_SCHEDULE), validate == 0 accepts any parsable sequence, such as one
+ * whose fused loops were already removed.  The zero-terminated text goes to buf (host memory, buf_len
+ * bytes, may be NULL); *needed receives its length including the terminator; CONST_ERR_WORKSPACE when
+ * the buffer was too small (the text is truncated).  Host only, no device work.
+ */
+const_status_t const_schedule_cin(const char *expression, const char *const *tree, int n_contractions,
+                                  const char *const *sparse_names, const int *const *mode_orders, int n_sparse,
+                                  const char *const *loop_orders, const const_extent_t *extents, int n_indices,
+                                  int validate, char *buf, int64_t buf_len, int64_t *needed);
+
+/*
  * Choose where the dense per-slice stage of a plan runs.  The last contraction of a TTMc, summed over
  * the fibres of a slice, is the contraction Y_i = U_J^T * T_J (K = fibres of the slice; the consumer
  * statement of the Fig. 4(b) structure regrouped).  enable != 0: const_execute runs it on the tensor

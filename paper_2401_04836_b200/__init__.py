@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     const_csf_bin_counts,
     const_plan_create,
     const_schedule_check,
+    const_schedule_cin,
     const_plan_reduced_order,
     const_plan_family,
     const_plan_set_tensor_stage,

@@ -65,6 +65,10 @@ def load_library():
                                       pp(pp(i32)), i32, pp(ctypes.c_char_p), pp(_Extent), i32, i32, pp(vp)]
     lib.const_schedule_check.argtypes = [ctypes.c_char_p, pp(ctypes.c_char_p), i32, pp(ctypes.c_char_p),
                                          pp(pp(i32)), i32, pp(ctypes.c_char_p), pp(_Extent), i32, pp(i32)]
+    lib.const_schedule_cin.argtypes = [ctypes.c_char_p, pp(ctypes.c_char_p), i32, pp(ctypes.c_char_p),
+                                       pp(pp(i32)), i32, pp(ctypes.c_char_p), pp(_Extent), i32, i32, ctypes.c_char_p,
+                                       i64, pp(i64)]
+    lib.const_schedule_cin.restype = i32
     lib.const_plan_reduced_order.argtypes = [vp, i32, pp(i32)]
     lib.const_plan_family.argtypes = [vp]
     lib.const_plan_family.restype = ctypes.c_char_p
@@ -260,6 +264,19 @@ def const_schedule_check(expression: str, tree: Sequence[str], mode_orders: Dict
     _check(lib.const_schedule_check(expression.encode(), tree_a, n_c, names_a, mo_a, n_s, loops_a, ext_a, n_e, red),
            "const_schedule_check")
     return list(red)
+
+
+def const_schedule_cin(expression: str, tree: Sequence[str], mode_orders: Dict[str, Sequence[int]],
+                       loop_orders: Sequence[str], extents: Dict[str, int], validate: bool = True) -> str:
+    """Host-only: concrete index notation (forall / where nest) of the schedule, Algorithm 1 of Sec. 4.2."""
+    lib = load_library()
+    tree_a, n_c, names_a, mo_a, n_s, loops_a, ext_a, n_e, _keep = _schedule_args(tree, mode_orders, loop_orders, extents)
+    need = ctypes.c_int64()
+    args = (expression.encode(), tree_a, n_c, names_a, mo_a, n_s, loops_a, ext_a, n_e, 1 if validate else 0)
+    _check(lib.const_schedule_cin(*args, None, 0, ctypes.byref(need)), "const_schedule_cin")
+    buf = ctypes.create_string_buffer(max(int(need.value), 1))
+    _check(lib.const_schedule_cin(*args, buf, len(buf), ctypes.byref(need)), "const_schedule_cin")
+    return buf.value.decode()
 
 
 def const_plan_create(expression: str, tree: Sequence[str], mode_orders: Dict[str, Sequence[int]],

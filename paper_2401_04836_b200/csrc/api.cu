@@ -2,6 +2,8 @@
 #include <cstring>
 #include <new>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 using namespace cb;
@@ -154,6 +156,26 @@ const_status_t const_schedule_check(const char *expression, const char *const *t
     if (rc == CONST_OK && reduced_orders)
         for (int c = 0; c < n_contractions; ++c) reduced_orders[c] = d.reduced_order[c];
     return rc;
+}
+
+const_status_t const_schedule_cin(const char *expression, const char *const *tree, int n_contractions,
+                                  const char *const *sparse_names, const int *const *mode_orders, int n_sparse,
+                                  const char *const *loop_orders, const const_extent_t *extents, int n_indices,
+                                  int validate, char *buf, int64_t buf_len, int64_t *needed) {
+    PlanDesc d;
+    const_status_t rc = parse_plan(expression, tree, n_contractions, sparse_names, mode_orders, n_sparse, loop_orders,
+                                   extents, n_indices, CONST_F32, d);
+    if (rc == CONST_OK && validate) rc = check_plan(d);
+    if (rc != CONST_OK) return rc;
+    const std::string text = schedule_cin(d);
+    if (needed) *needed = (int64_t)text.size() + 1;
+    if (buf && buf_len > 0) {
+        const size_t n = std::min<size_t>(text.size(), (size_t)buf_len - 1);
+        std::memcpy(buf, text.data(), n);
+        buf[n] = 0;
+        if (n < text.size()) return CONST_ERR_WORKSPACE;
+    }
+    return CONST_OK;
 }
 
 const_status_t const_plan_reduced_order(const const_plan_t *h, int contraction, int *order) {
