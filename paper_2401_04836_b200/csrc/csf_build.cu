@@ -436,6 +436,8 @@ struct CsfArrays {
     int bits[kMaxOrder];
 };
 
+// ORDER is a template parameter so that the per-level arrays are indexed by constants and stay in registers.
+template <int ORDER>
 __global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__restrict__ keys, int64_t n, LevelShifts ls,
                                                          const uint32_t *__restrict__ block_base, CsfArrays out) {
     __shared__ uint32_t wcnt[kCpThreads / 32][kCpLevels];
@@ -460,7 +462,7 @@ __global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__rest
         run[l] = block_base[(int64_t)blockIdx.x * kCpLevels + l];
         for (int w = 0; w < warp; ++w) run[l] += wcnt[w][l];
     }
-    const int leaf = ls.order - 1;
+    constexpr int leaf = ORDER - 1;
     const unsigned below = (1u << lane) - 1u;
 #pragma unroll
     for (int it = 0; it < kCpIters; ++it) {
@@ -481,6 +483,16 @@ __global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__rest
         }
 #pragma unroll
         for (int l = 0; l < kCpLevels; ++l) run[l] += __popc(bal[it][l]);
+    }
+}
+
+inline void launch_csf_scatter(int order, int64_t blocks, const uint64_t *keys, int64_t n, const LevelShifts &ls,
+                               const uint32_t *block_base, const CsfArrays &out, cudaStream_t stream) {
+    switch (order) {
+        case 1: csf_scatter<1><<<(unsigned)blocks, kCpThreads, 0, stream>>>(keys, n, ls, block_base, out); break;
+        case 2: csf_scatter<2><<<(unsigned)blocks, kCpThreads, 0, stream>>>(keys, n, ls, block_base, out); break;
+        case 3: csf_scatter<3><<<(unsigned)blocks, kCpThreads, 0, stream>>>(keys, n, ls, block_base, out); break;
+        default: csf_scatter<4><<<(unsigned)blocks, kCpThreads, 0, stream>>>(keys, n, ls, block_base, out); break;
     }
 }
 
@@ -923,7 +935,7 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
                 arr.crd[l] = csf->crd[l];
             }
             if (nnz > 0)
-                CB_LAUNCH("csf_scatter", stream, csf_scatter<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, arr));
+                CB_LAUNCH("csf_scatter", stream, launch_csf_scatter(order, cp_blocks, keys, nnz, ls, block_counts, arr, stream));
             LevelSizes sz;
             sz.order = order;
             for (int l = 0; l < kMaxOrder; ++l) sz.n[l] = csf->n[l];
@@ -1052,7 +1064,7 @@ const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nn
         arr.crd[l] = l < order ? crd_out[l] : nullptr;
         arr.bits[l] = kl.bits[l];
     }
-    if (nnz > 0) csf_scatter<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, arr);
+    if (nnz > 0) launch_csf_scatter(order, cp_blocks, keys, nnz, ls, block_counts, arr, stream);
     csf_finish<<<1, 32, 0, stream>>>(arr, sz);
     CB_CUDA(cudaGetLastError());
     if (level_sizes)
