@@ -367,6 +367,22 @@ __device__ __forceinline__ void node_flags(const uint64_t *__restrict__ keys, in
     }
 }
 
+// the same flags from a key the caller already holds; `carry` = the element before `base` (unused when base == 0)
+__device__ __forceinline__ void node_flags_of(int64_t n, int64_t base, int lane, const LevelShifts &ls, uint64_t key,
+                                              uint64_t carry, unsigned ballots[kCpLevels]) {
+    const int64_t e = base + lane;
+    const bool in = e < n;
+    uint64_t prev = __shfl_up_sync(0xffffffffu, key, 1);
+    if (lane == 0) prev = carry;
+    const bool first = (e == 0);
+#pragma unroll
+    for (int l = 0; l < kCpLevels; ++l) {
+        bool f = false;
+        if (l < ls.order - 1) f = in && (first || (key >> ls.shift[l]) != (prev >> ls.shift[l]));
+        ballots[l] = __ballot_sync(0xffffffffu, f);
+    }
+}
+
 __global__ void __launch_bounds__(kCpThreads) csf_count(const uint64_t *__restrict__ keys, int64_t n, LevelShifts ls,
                                                        uint32_t *__restrict__ block_counts, int32_t *status) {
     __shared__ uint32_t sh[kCpLevels];
@@ -445,11 +461,18 @@ __global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__rest
     uint64_t key[kCpIters];
     unsigned bal[kCpIters][kCpLevels];
     uint32_t cnt[kCpLevels] = {0, 0, 0};
+    // the warp's kCpIters * 32 consecutive keys and the one in front of them, all requested before the first is used
+    const int64_t warp_base = (int64_t)blockIdx.x * kCpTile + (int64_t)warp * kCpIters * 32;
+    uint64_t carry = warp_base > 0 && warp_base <= n ? keys[warp_base - 1] : 0ull;
 #pragma unroll
     for (int it = 0; it < kCpIters; ++it) {
-        int64_t base = (int64_t)blockIdx.x * kCpTile + (warp * kCpIters + it) * 32;
-        bool dup;
-        node_flags(keys, n, base, lane, ls, key[it], bal[it], dup);
+        const int64_t e = warp_base + it * 32 + lane;
+        key[it] = e < n ? keys[e] : 0ull;
+    }
+#pragma unroll
+    for (int it = 0; it < kCpIters; ++it) {
+        node_flags_of(n, warp_base + it * 32, lane, ls, key[it], carry, bal[it]);
+        carry = __shfl_sync(0xffffffffu, key[it], 31);
 #pragma unroll
         for (int l = 0; l < kCpLevels; ++l) cnt[l] += __popc(bal[it][l]);
     }
