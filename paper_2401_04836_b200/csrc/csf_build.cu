@@ -64,8 +64,12 @@ __global__ void __launch_bounds__(256) pack_hist(PackArgs a, int64_t nnz, DigitP
             key |= (uint64_t)c << a.shift[l];
         }
         keys[e] = key;
-        for (int p = 0; p < dp.passes; ++p)
-            atomicAdd(&sh[p * kRsMaxBins + ((unsigned)(key >> dp.shift[p]) & ((1u << dp.bits[p]) - 1u))], 1u);
+        // unrolled over the maximum so that the plan is read with constant indices (a runtime index would
+        // send the parameter arrays through local memory, ten loads per nonzero)
+#pragma unroll
+        for (int p = 0; p < kMaxPasses; ++p)
+            if (p < dp.passes)
+                atomicAdd(&sh[p * kRsMaxBins + ((unsigned)(key >> dp.shift[p]) & ((1u << dp.bits[p]) - 1u))], 1u);
     }
     if (bad) report(status, CONST_ERR_COORD_RANGE);
     __syncthreads();
