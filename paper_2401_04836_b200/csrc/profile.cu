@@ -55,6 +55,14 @@ const_status_t const_profile_enable(int on) {
     g_on = on != 0;
     for (Span &s : g_spans) { g_pool.push_back(s.a); g_pool.push_back(s.b); }
     g_spans.clear();
+    // events are created here, not at the first launches that need them: creating one can take a
+    // millisecond on some hosts, which would land inside the region that is being timed
+    constexpr size_t kPrepared = 4096;
+    while (g_on && g_pool.size() < kPrepared) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess || !e) break;
+        g_pool.push_back(e);
+    }
     return CONST_OK;
 }
 
