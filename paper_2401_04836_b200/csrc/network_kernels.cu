@@ -48,6 +48,7 @@ struct Stage {                 // shared-memory staging area of one sweep
     Rec *recs;                 // [RB]
     int32_t *fpos;             // [FPMAX + 1] first nonzero of every staged fibre
     int32_t *fcrd;             // [FPMAX]     level-1 coordinate of every staged fibre
+    int32_t *first;            // staged fibre that holds the first nonzero of the current chunk
 };
 
 // Calls body(fibre, coordinate, records, count) once for every piece of every fibre in [fA, fB) of
@@ -73,12 +74,12 @@ __device__ __forceinline__ void sweep(const Csf3d &x, int32_t fA, int32_t fB, co
                 r.v = __ldg(x.vals + c0 + e);
                 st.recs[e] = r;
             }
+            // the staged fibre that holds nonzero c0: every thread tests its candidates (exactly one fits),
+            // which costs a few instructions where a search per thread costs a dependent chain
+            for (int e = threadIdx.x; e < nf; e += kThreads)
+                if (st.fpos[e] <= c0 && c0 < st.fpos[e + 1]) *st.first = e;
             __syncthreads();
-            int lo = 0, hi = nf - 1;                       // staged fibre that holds nonzero c0
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (st.fpos[mid] <= c0) lo = mid; else hi = mid - 1;
-            }
+            const int lo = *st.first;
             for (int f = lo + g; f < nf; f += NG) {
                 const int32_t a = st.fpos[f], b = st.fpos[f + 1];
                 if (a >= c1) break;
@@ -107,6 +108,8 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
     __shared__ int32_t w_pos[LT + 1];              // first fibre of every l node of the tile
     __shared__ int32_t w_l[LT];                    // l of those nodes, relative to the tile
     __shared__ int32_t w_nodes;
+    __shared__ int32_t s_first;
+    st.first = &s_first;
 
     const int strip = blockIdx.x, l0 = blockIdx.y * LT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
