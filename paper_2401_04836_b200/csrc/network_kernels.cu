@@ -29,7 +29,7 @@ namespace {
 
 constexpr int LT = 8;          // l values per block
 constexpr int kThreads = 512;
-constexpr int RB = 2048;       // records staged per chunk
+constexpr int RB = 2048;       // records staged per chunk (a multiple of the block size)
 constexpr int FPMAX = 1024;    // fibre descriptors staged per batch
 
 struct Csf3d {
@@ -65,20 +65,37 @@ __device__ __forceinline__ void sweep(const Csf3d &x, int32_t fA, int32_t fB, co
         for (int e = threadIdx.x; e < nf; e += kThreads) st.fcrd[e] = __ldg(x.crd1 + fb0 + e);
         __syncthreads();
         const int32_t pA = st.fpos[0], pB = st.fpos[nf];
+        // the records of a chunk are requested one chunk ahead and wait in registers while the chunk
+        // before them is multiplied, so the global-memory latency of the staging is hidden
+        constexpr int PER = RB / kThreads;
+        int32_t pc[PER];
+        double pv[PER];
+        auto request = [&](int32_t c0) {
+#pragma unroll
+            for (int q = 0; q < PER; ++q) {
+                const int32_t p = c0 + threadIdx.x + q * kThreads;
+                pc[q] = 0;
+                pv[q] = 0.0;
+                if (p < pB) { pc[q] = __ldg(x.crd2 + p); pv[q] = __ldg(x.vals + p); }
+            }
+        };
+        request(pA);
         for (int32_t c0 = pA; c0 < pB; c0 += RB) {
             const int32_t c1 = c0 + RB < pB ? c0 + RB : pB;
-            for (int e = threadIdx.x; e < c1 - c0; e += kThreads) {
+#pragma unroll
+            for (int q = 0; q < PER; ++q) {
                 Rec r;
-                r.c = __ldg(x.crd2 + c0 + e);
+                r.c = pc[q];
                 r.pad = 0;
-                r.v = __ldg(x.vals + c0 + e);
-                st.recs[e] = r;
+                r.v = pv[q];
+                st.recs[threadIdx.x + q * kThreads] = r;
             }
             // the staged fibre that holds nonzero c0: every thread tests its candidates (exactly one fits),
             // which costs a few instructions where a search per thread costs a dependent chain
             for (int e = threadIdx.x; e < nf; e += kThreads)
                 if (st.fpos[e] <= c0 && c0 < st.fpos[e + 1]) *st.first = e;
             __syncthreads();
+            if (c1 < pB) request(c1);
             const int lo = *st.first;
             for (int f = lo + g; f < nf; f += NG) {
                 const int32_t a = st.fpos[f], b = st.fpos[f + 1];
