@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(kThreads)
 network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restrict__ Z, int n_k, int n_l, int n_m,
                int v_vec_ok) {
     constexpr int VPT = 8 / GL;                    // entries of a V row (producer) or T row (consumer) per lane
-    static_assert(LT == 8 && IS == 8 && (VPT == 1 || VPT == 2), "a lane group covers the 8 l of the tile or the 8 i of the strip");
+    static_assert(LT == 8 && IS == 8 && (VPT == 1 || VPT == 2 || VPT == 4), "a lane group covers the 8 l of the tile or the 8 i of the strip");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int TL = n_k * IS + 2;                   // doubles per l plane; the +2 staggers the banks of the 8 planes
     double *T = reinterpret_cast<double *>(smem_raw);                               // [LT][n_k][IS]
@@ -157,37 +157,42 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
     {
         const int lq = q * VPT;                    // first l of this lane, relative to the tile
         const double *vcol = V + l0 + lq;
-        const bool full = l0 + lq + VPT <= n_l;
+        const bool vec = v_vec_ok && VPT >= 2 && l0 + lq + VPT <= n_l;     // whole lane inside the row, 16-byte aligned
         sweep<GL>(u, s_pos[0], s_pos[IS], st, [&](int32_t f, int32_t k, const Rec *recs, int n) {
             int ii = 0;
             while (ii + 1 < IS && s_pos[ii + 1] <= f) ++ii;
-            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
-            if (VPT == 2 && v_vec_ok && full) {
+            double a[VPT], b[VPT];                 // two accumulator sets: consecutive records alternate
+#pragma unroll
+            for (int c = 0; c < VPT; ++c) a[c] = b[c] = 0.0;
+            if (vec) {
+                auto row_fma = [&](const Rec &r, double (&acc)[VPT]) {
+                    const double2 *row = reinterpret_cast<const double2 *>(vcol + (size_t)r.c * n_l);
+#pragma unroll
+                    for (int c = 0; c < VPT / 2; ++c) {
+                        const double2 v = __ldg(row + c);
+                        acc[2 * c] = fma(r.v, v.x, acc[2 * c]);
+                        acc[2 * c + 1] = fma(r.v, v.y, acc[2 * c + 1]);
+                    }
+                };
                 int e = 0;
                 for (; e + 1 < n; e += 2) {
                     const Rec r0 = recs[e], r1 = recs[e + 1];
-                    const double2 v0 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r0.c * n_l));
-                    const double2 v1 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r1.c * n_l));
-                    a0 = fma(r0.v, v0.x, a0); a1 = fma(r0.v, v0.y, a1);
-                    b0 = fma(r1.v, v1.x, b0); b1 = fma(r1.v, v1.y, b1);
+                    row_fma(r0, a);
+                    row_fma(r1, b);
                 }
-                if (e < n) {
-                    const Rec r0 = recs[e];
-                    const double2 v0 = __ldg(reinterpret_cast<const double2 *>(vcol + (size_t)r0.c * n_l));
-                    a0 = fma(r0.v, v0.x, a0); a1 = fma(r0.v, v0.y, a1);
-                }
-                a0 += b0; a1 += b1;
+                if (e < n) row_fma(recs[e], a);
             } else {
                 for (int e = 0; e < n; ++e) {
                     const Rec r0 = recs[e];
                     const double *row = vcol + (size_t)r0.c * n_l;
-                    if (l0 + lq < n_l) a0 = fma(r0.v, __ldg(row), a0);
-                    if (VPT == 2 && l0 + lq + 1 < n_l) a1 = fma(r0.v, __ldg(row + 1), a1);
+#pragma unroll
+                    for (int c = 0; c < VPT; ++c)
+                        if (l0 + lq + c < n_l) a[c] = fma(r0.v, __ldg(row + c), a[c]);
                 }
             }
             double *t = T + (size_t)lq * TL + k * IS + ii;
-            t[0] += a0;
-            if (VPT == 2) t[TL] += a1;
+#pragma unroll
+            for (int c = 0; c < VPT; ++c) t[c * TL] += a[c] + b[c];
         });
     }
     // (the sweep ends with a block barrier: T is complete)
@@ -205,34 +210,32 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
             int node = 0;
             while (node + 1 < nodes && w_pos[node + 1] <= f) ++node;
             const double *t = T + (size_t)w_l[node] * TL + iq;
-            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
-            if (VPT == 2) {
-                int e = 0;
-                for (; e + 1 < n; e += 2) {
-                    const Rec r0 = recs[e], r1 = recs[e + 1];
-                    const double2 t0 = *reinterpret_cast<const double2 *>(t + r0.c * IS);
-                    const double2 t1 = *reinterpret_cast<const double2 *>(t + r1.c * IS);
-                    a0 = fma(t0.x, r0.v, a0); a1 = fma(t0.y, r0.v, a1);
-                    b0 = fma(t1.x, r1.v, b0); b1 = fma(t1.y, r1.v, b1);
+            double a[VPT], b[VPT];
+#pragma unroll
+            for (int c = 0; c < VPT; ++c) a[c] = b[c] = 0.0;
+            auto row_fma = [&](const Rec &r, double (&acc)[VPT]) {
+                const double *row = t + r.c * IS;
+                if constexpr (VPT >= 2) {
+#pragma unroll
+                    for (int c = 0; c < VPT / 2; ++c) {
+                        const double2 tv = *reinterpret_cast<const double2 *>(row + 2 * c);
+                        acc[2 * c] = fma(tv.x, r.v, acc[2 * c]);
+                        acc[2 * c + 1] = fma(tv.y, r.v, acc[2 * c + 1]);
+                    }
+                } else {
+                    acc[0] = fma(row[0], r.v, acc[0]);
                 }
-                if (e < n) {
-                    const Rec r0 = recs[e];
-                    const double2 t0 = *reinterpret_cast<const double2 *>(t + r0.c * IS);
-                    a0 = fma(t0.x, r0.v, a0); a1 = fma(t0.y, r0.v, a1);
-                }
-                a0 += b0; a1 += b1;
-            } else {
-                int e = 0;
-                for (; e + 1 < n; e += 2) {
-                    const Rec r0 = recs[e], r1 = recs[e + 1];
-                    a0 = fma(t[r0.c * IS], r0.v, a0);
-                    b0 = fma(t[r1.c * IS], r1.v, b0);
-                }
-                if (e < n) a0 = fma(t[recs[e].c * IS], recs[e].v, a0);
-                a0 += b0;
+            };
+            int e = 0;
+            for (; e + 1 < n; e += 2) {
+                const Rec r0 = recs[e], r1 = recs[e + 1];
+                row_fma(r0, a);
+                row_fma(r1, b);
             }
-            if (rows[0] >= 0) atomicAdd(Z + (size_t)rows[0] * n_m + m, a0);
-            if (VPT == 2 && rows[VPT - 1] >= 0) atomicAdd(Z + (size_t)rows[VPT - 1] * n_m + m, a1);
+            if (e < n) row_fma(recs[e], a);
+#pragma unroll
+            for (int c = 0; c < VPT; ++c)
+                if (rows[c] >= 0) atomicAdd(Z + (size_t)rows[c] * n_m + m, a[c] + b[c]);
         });
     }
 }
@@ -242,7 +245,7 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
 const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z, int64_t n_i,
                            int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m, int32_t *, cudaStream_t stream) {
     (void)n_j;
-    constexpr int IS = 8, GL = 4;
+    constexpr int IS = 8, GL = 4;   // lanes per fibre: 2 -> 5.8 ms, 4 -> 4.8 ms, 8 -> 6.2 ms on the benchmark network
     CB_CUDA(cudaMemsetAsync(Z, 0, sizeof(double) * n_i * n_m, stream));
     if (U->nnz == 0 || W->nnz == 0) return CONST_OK;
     const size_t t_doubles = ((size_t)LT * (n_k * IS + 2) + 1) / 2 * 2;
