@@ -46,7 +46,7 @@ struct const_csf {
     int32_t *slice_ptr = nullptr;      // [n0 + 1] leaf offset of every root-level slice
     int32_t *light_list = nullptr;     // [n_light] slice ids handled one per warp
     cb::WorkItem *items = nullptr;     // [n_items]
-    int32_t *bin_scratch = nullptr;    // [2 * (n0 + 1) + 8] scan outputs
+    int32_t *bin_scratch = nullptr;    // [2 * (n0 + 1) + 8 + 64] scan outputs, size-class bases and fill counters
     int64_t n_light = 0, n_heavy = 0, n_giant = 0, n_items = 0;
     int64_t light_max = 0, heavy_max = 0, chunk = 0;
     cudaStream_t stream = nullptr;

@@ -551,14 +551,22 @@ __global__ void bin_slice_ptr(ChainPtrs c, int64_t n0, int32_t *__restrict__ sli
     slice_ptr[s] = leaf_of_fiber(c, c.pos[1][s]);
 }
 
-// Single-block scan over slices: per-slice work-item offset and light-list index; totals in out[0..4).
+// Light slices are listed by falling size class (class = floor(log2(nonzeros))), so that the slices that
+// share a block are about equally large and the largest start first.  kBinClasses classes; totals[8 + d] =
+// first list position of class d (d = 0: largest), totals[8 + kBinClasses + d] = fill counter, cleared.
+constexpr int kBinClasses = 32;
+__device__ __forceinline__ int light_class(int64_t z) { return 31 - (63 - __clzll((unsigned long long)(z > 0 ? z : 1))); }
+
+// Single-block scan over slices: per-slice work-item offset; totals in out[0..4), class bases behind them.
 __global__ void __launch_bounds__(1024) bin_scan(const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t light_max,
                                                  int64_t heavy_max, int64_t chunk, int32_t *__restrict__ item_off,
                                                  int32_t *__restrict__ light_idx, int32_t *__restrict__ totals) {
     __shared__ uint32_t wsum[32][2];
     __shared__ uint32_t carry[4];      // items, light, heavy, giant
+    __shared__ uint32_t cls[kBinClasses];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x < 4) carry[threadIdx.x] = 0;
+    if (threadIdx.x < kBinClasses) cls[threadIdx.x] = 0;
     __syncthreads();
     for (int64_t base = 0; base < n0; base += 1024) {
         int64_t s = base + threadIdx.x;
@@ -566,7 +574,7 @@ __global__ void __launch_bounds__(1024) bin_scan(const int32_t *__restrict__ sli
         uint32_t is_heavy = 0, is_giant = 0;
         if (s < n0) {
             int64_t z = (int64_t)slice_ptr[s + 1] - slice_ptr[s];
-            if (z <= light_max) v[1] = 1;
+            if (z <= light_max) { v[1] = 1; atomicAdd(&cls[light_class(z)], 1u); }
             else if (z <= heavy_max) { v[0] = 1; is_heavy = 1; }
             else { v[0] = (uint32_t)((z + chunk - 1) / chunk); is_giant = 1; }
         }
@@ -595,16 +603,27 @@ __global__ void __launch_bounds__(1024) bin_scan(const int32_t *__restrict__ sli
         __syncthreads();
     }
     if (threadIdx.x < 4) totals[threadIdx.x] = (int32_t)carry[threadIdx.x];
+    if (threadIdx.x == 0) {
+        uint32_t run = 0;
+        for (int d = 0; d < kBinClasses; ++d) {
+            totals[8 + d] = (int32_t)run;
+            totals[8 + kBinClasses + d] = 0;
+            run += cls[d];
+        }
+    }
 }
 
 __global__ void bin_fill(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t light_max,
                          int64_t heavy_max, const int32_t *__restrict__ item_off,
-                         const int32_t *__restrict__ light_idx, WorkItem *__restrict__ items,
+                         int32_t *__restrict__ class_base, WorkItem *__restrict__ items,
                          int32_t *__restrict__ light_list) {
     int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n0) return;
     const int64_t z = (int64_t)slice_ptr[s + 1] - slice_ptr[s];
-    if (z <= light_max) light_list[light_idx[s]] = (int32_t)s;
+    if (z <= light_max) {       // any order inside a class will do: slices are independent of one another
+        const int d = light_class(z);
+        light_list[class_base[d] + atomicAdd(&class_base[kBinClasses + d], 1)] = (int32_t)s;
+    }
     else if (z <= heavy_max) items[item_off[s]] = WorkItem{(int32_t)s, c.pos[1][s], c.pos[1][s + 1], kItemBlock};
 }
 
@@ -881,7 +900,7 @@ const_status_t csf_rebin(const_csf *csf, cudaStream_t stream) {
     CB_CUDA(pool_alloc((void **)&csf->items, sizeof(WorkItem) * std::max<int64_t>(csf->n_items, 1), stream));
     CB_CUDA(pool_alloc((void **)&csf->light_list, sizeof(int32_t) * std::max<int64_t>(csf->n_light, 1), stream));
     CB_LAUNCH("bin_fill", stream, bin_fill<<<(unsigned)((n0 + 255) / 256), 256, 0, stream>>>(c, csf->slice_ptr, n0, csf->light_max, csf->heavy_max,
-                                                              item_off, light_idx, csf->items, csf->light_list));
+                                                              item_off, totals + 8, csf->items, csf->light_list));
     if (hg_items > 0)
         CB_LAUNCH("bin_fill_chunks", stream, bin_fill_chunks<<<(unsigned)((hg_items + 127) / 128), 128, 0, stream>>>(
                       c, csf->slice_ptr, n0, csf->heavy_max, csf->chunk, item_off, hg_items, csf->items));
@@ -974,7 +993,7 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             // per-slice leaf offsets and the default work lists
             const int64_t n0 = csf->n[0];
             CB_CUDA(pool_alloc((void **)&csf->slice_ptr, sizeof(int32_t) * (n0 + 1), stream));
-            CB_CUDA(pool_alloc((void **)&csf->bin_scratch, sizeof(int32_t) * (2 * (n0 + 1) + 8), stream));
+            CB_CUDA(pool_alloc((void **)&csf->bin_scratch, sizeof(int32_t) * (2 * (n0 + 1) + 8 + 2 * kBinClasses), stream));
             ChainPtrs c;
             c.order = order;
             for (int l = 0; l < kMaxOrder; ++l) c.pos[l] = csf->pos[l];
