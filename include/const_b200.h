@@ -14,7 +14,8 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - The caller owns COO inputs, dense factors and outputs.  The library owns CSF arrays, work lists
  *     and scratch (stream-ordered allocations on the given stream) until const_destroy.
- *   - Dense operands and outputs are row-major in the index order written in the expression.
+ *   - Dense operands and outputs are row-major in the index order written in the expression, and their
+ *     base addresses are 16-byte aligned (rows are read and written with 128-bit accesses).
  *   - Every function returns a const_status_t; on error no output handle is produced.
  */
 #ifndef CONST_B200_H
@@ -65,11 +66,13 @@ typedef struct { const char *name; const const_csf_t *csf; const void *dense_dev
  * The coordinate tuple is packed into one 64-bit key (sum of ceil(log2 extent) over modes must be
  * <= 64), radix-sorted with its value, then each level is compressed with a flag/scan/scatter pass.
  * Per-slice nonzero counts and the light / heavy / giant work lists used by const_execute are built
- * here as well.
+ * here as well (on the device; the host does not wait for them).
  *
  * Errors: CONST_ERR_COORD_RANGE, CONST_ERR_DUPLICATE_COORD (both detected on the device; the call
- * synchronises the stream once to read sizes and status), CONST_ERR_UNSUPPORTED for nnz >= 2^31 - 1
- * or a key wider than 64 bits, CONST_ERR_INVALID_ARG, CONST_ERR_CUDA.
+ * waits for the stream once, after the sort, to read the level sizes and the status),
+ * CONST_ERR_UNSUPPORTED for nnz >= 2^31 - 1 or a key wider than 64 bits, CONST_ERR_TIMEOUT when a
+ * bounded device-side wait of the sort gave up (nothing is stored then), CONST_ERR_INVALID_ARG,
+ * CONST_ERR_CUDA.  Safe to call from several host threads at once.
  */
 const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz,
                                const int32_t *const *coords_dev, const void *vals_dev, const_dtype_t dtype,
@@ -98,6 +101,9 @@ const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz,
  *
  * The first call on each device looks up the device address of that array (one
  * cudaGetSymbolAddress with that device current); make that first call outside any stream capture.
+ * With CUDA's lazy module loading that first call is also the moment the driver loads the kernels and
+ * places the array on the device, so "obtains no device memory" holds from the second call on: make
+ * one warm-up call per device at start-up, while allocating is still allowed.
  * All calls share the array and it keeps whatever the previous call left in it; the call clears the
  * parts that must start at zero.  Two calls whose GPU work overlaps (different streams, or different
  * host threads) race on it: serialise them.  Like const_csf_build, the call synchronises the stream
@@ -125,9 +131,22 @@ const_status_t const_csf_values(const const_csf_t *csf, const void **vals, int64
  */
 const_status_t const_csf_set_bins(const_csf_t *csf, int64_t light_max_nnz, int64_t heavy_max_nnz,
                                   int64_t chunk_nnz, void *stream);
-/* Number of slices in each bin and of thread-block work items; any pointer may be NULL. */
+/* Number of slices in each bin and of thread-block work items; any pointer may be NULL.  The counts live on
+ * the device; the first request after a (re)binning waits for the stream that did it. */
 const_status_t const_csf_bin_counts(const const_csf_t *csf, int64_t *n_light, int64_t *n_heavy,
                                     int64_t *n_giant, int64_t *n_items);
+/*
+ * Borrowed device pointers of the work lists, for checking the load balancer (valid until the next
+ * const_csf_set_bins or const_destroy; any pointer may be NULL):
+ *   slice_ptr[n_0 + 1]   leaf offset of every root-level slice (slice s holds leaves [slice_ptr[s], slice_ptr[s+1]));
+ *   light_list[n_light]  the light slices, by falling size class floor(log2(nonzeros));
+ *   items[n_items][4]    one record {slice, f0, f1, kind} of four int32 per thread block:
+ *                          kind 1: heavy slice `slice`, all its level-1 nodes [f0, f1);
+ *                          kind 2: level-1 nodes [f0, f1) of giant slice `slice` (its chunks tile the slice);
+ *                          kind 0: entries [slice, slice + f0) of light_list, one slice per warp.
+ */
+const_status_t const_csf_work_lists(const const_csf_t *csf, const int32_t **slice_ptr, const int32_t **light_list,
+                                    int64_t *n_light, const int32_t **items, int64_t *n_items);
 
 /*
  * Check a schedule and bind it to a kernel family (Sec. 3.1 input/output; Sec. 3.2 constraints;
@@ -188,7 +207,10 @@ const char *const_plan_family(const const_plan_t *plan);
  * Run the fused contraction tree (Fig. 4(b) / Fig. 5 structure).  `operands` binds every input name
  * of the expression to a CSF handle or a dense device array; CSF handles must have been built with
  * the mode order and dtype the plan was created with.  out_dev is overwritten (it is zeroed first:
- * "R[*] = 0" precedes the nest).  Asynchronous on `stream`; no host synchronisation.
+ * "R[*] = 0" precedes the nest).  Asynchronous on `stream`; no host synchronisation, the first call
+ * included (the plan's status word is allocated and cleared in stream order then).  A plan stays on
+ * the device of its first execute.  Every dense operand and out_dev must be 16-byte aligned
+ * (CONST_ERR_INVALID_ARG otherwise, before anything is launched).
  * Partial results of split slices are combined with floating-point atomics, so results can differ
  * in the last bits between runs.
  */
@@ -235,6 +257,16 @@ const_status_t const_last_device_status(const_plan_t *plan, void *stream);
 void const_destroy(void *handle);
 
 const char *const_status_string(const_status_t status);
+
+/*
+ * Test hook for the bounded device-side waits (the look-back of the radix sort, the mbarrier wait of the
+ * tensor-core stage).  what = 0: number of polls after which a wait gives up (0 restores the defaults);
+ * what = 1: value != 0 withholds the signal those waits wait for -- sort tiles do not publish their
+ * counts, the tensor-core stage issues and commits nothing -- so that every such wait runs out, the
+ * kernel records CONST_ERR_TIMEOUT, skips its stores and returns normally.  Process-wide; not for
+ * production use.  CONST_ERR_INVALID_ARG for an unknown `what` or a value outside [0, 2^31).
+ */
+const_status_t const_debug_set(int what, int64_t value);
 
 /*
  * Per-kernel timing (off by default).  While enabled, every kernel the library launches is

@@ -16,6 +16,8 @@ from .binding import (  # noqa: F401
     const_csf_values,
     const_csf_set_bins,
     const_csf_bin_counts,
+    const_csf_work_lists,
+    const_debug_set,
     const_plan_create,
     const_schedule_check,
     const_schedule_cin,

@@ -61,6 +61,10 @@ def load_library():
     lib.const_csf_values.argtypes = [vp, pp(vp), pp(i64)]
     lib.const_csf_set_bins.argtypes = [vp, i64, i64, i64, vp]
     lib.const_csf_bin_counts.argtypes = [vp, pp(i64), pp(i64), pp(i64), pp(i64)]
+    lib.const_csf_work_lists.argtypes = [vp, pp(vp), pp(vp), pp(i64), pp(vp), pp(i64)]
+    lib.const_csf_work_lists.restype = i32
+    lib.const_debug_set.argtypes = [i32, i64]
+    lib.const_debug_set.restype = i32
     lib.const_plan_create.argtypes = [ctypes.c_char_p, pp(ctypes.c_char_p), i32, pp(ctypes.c_char_p),
                                       pp(pp(i32)), i32, pp(ctypes.c_char_p), pp(_Extent), i32, i32, pp(vp)]
     lib.const_schedule_check.argtypes = [ctypes.c_char_p, pp(ctypes.c_char_p), i32, pp(ctypes.c_char_p),
@@ -240,6 +244,25 @@ def const_csf_bin_counts(csf: CsfHandle) -> Dict[str, int]:
     return {"light": a.value, "heavy": b.value, "giant": c.value, "items": d.value}
 
 
+def const_csf_work_lists(csf: CsfHandle):
+    """Copies of the load balancer's lists: (slice_ptr [n0+1], light_list [n_light], items [n_items, 4]) as int32 CUDA tensors."""
+    import torch
+    lib = load_library()
+    sp, ll, it = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()
+    n_light, n_items, n0 = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(lib.const_csf_work_lists(csf.ptr, ctypes.byref(sp), ctypes.byref(ll), ctypes.byref(n_light), ctypes.byref(it),
+                                    ctypes.byref(n_items)), "const_csf_work_lists")
+    _check(lib.const_csf_level(csf.ptr, 0, None, None, ctypes.byref(n0)), "const_csf_level")
+    return (_dev_to_torch(sp.value, n0.value + 1 if n0.value else 0, torch.int32),
+            _dev_to_torch(ll.value, n_light.value, torch.int32),
+            _dev_to_torch(it.value, 4 * n_items.value, torch.int32).reshape(-1, 4))
+
+
+def const_debug_set(what: int, value: int) -> None:
+    """Test hook: limits of the bounded device-side waits (see the header)."""
+    _check(load_library().const_debug_set(int(what), int(value)), "const_debug_set")
+
+
 def _schedule_args(tree, mode_orders, loop_orders, extents):
     n_c = len(tree)
     if len(loop_orders) != n_c:
@@ -283,20 +306,10 @@ def const_plan_create(expression: str, tree: Sequence[str], mode_orders: Dict[st
                       loop_orders: Sequence[str], extents: Dict[str, int], dtype: int) -> PlanHandle:
     """Host-only: parses and checks the schedule, binds a kernel family.  Needs no GPU."""
     lib = load_library()
-    n_c = len(tree)
-    if len(loop_orders) != n_c:
-        raise ValueError("one loop order per contraction")
-    tree_a = (ctypes.c_char_p * n_c)(*[t.encode() for t in tree])
-    loops_a = (ctypes.c_char_p * n_c)(*[s.encode() for s in loop_orders])
-    names = list(mode_orders)
-    names_a = (ctypes.c_char_p * max(len(names), 1))(*[n.encode() for n in names])
-    mo_arrays = [(ctypes.c_int * len(mode_orders[n]))(*[int(x) for x in mode_orders[n]]) for n in names]
-    mo_a = (ctypes.POINTER(ctypes.c_int) * max(len(names), 1))(
-        *[ctypes.cast(a, ctypes.POINTER(ctypes.c_int)) for a in mo_arrays])
-    ext_a = (_Extent * len(extents))(*[_Extent(k.encode(), int(v)) for k, v in extents.items()])
+    tree_a, n_c, names_a, mo_a, n_s, loops_a, ext_a, n_e, _keep = _schedule_args(tree, mode_orders, loop_orders, extents)
     out = ctypes.c_void_p()
-    st = lib.const_plan_create(expression.encode(), tree_a, n_c, names_a, mo_a, len(names), loops_a, ext_a,
-                               len(extents), int(dtype), ctypes.byref(out))
+    st = lib.const_plan_create(expression.encode(), tree_a, n_c, names_a, mo_a, n_s, loops_a, ext_a, n_e,
+                               int(dtype), ctypes.byref(out))
     _check(st, "const_plan_create")
     return PlanHandle(out.value)
 

@@ -11,7 +11,7 @@ LIB_PATH = os.path.join(_HERE, "libconst_b200.so")
 SOURCES = ["api.cu", "plan.cpp", "cin.cpp", "csf_build.cu", "chain_kernels.cu", "ttmc4_kernel.cu", "ttmc4_tc_kernel.cu", "chain3_tc_kernel.cu", "network_kernels.cu", "profile.cu"]
 HEADERS = ["common.cuh", "umma.cuh", "plan.h", os.path.join("..", "..", "include", "const_b200.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 
 
 def _nvcc() -> str:
@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     objdir = os.path.join(_HERE, "_build")
     os.makedirs(objdir, exist_ok=True)
     nvcc = _nvcc()
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = list(NVCC_FLAGS)
     if verbose:
         flags += ["-Xptxas", "-v"]
     procs = []

@@ -1,8 +1,8 @@
 // C-ABI entry points (include/const_b200.h): argument checking, handle management, dispatch.
+#include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <new>
-
-#include <algorithm>
 
 #include "common.cuh"
 
@@ -39,7 +39,15 @@ bool csf_matches(const const_csf *c, const PlanDesc &d, const std::string &name,
     return true;
 }
 
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+std::atomic<int> g_spin_limit{0}, g_withhold{0};
+
 }  // namespace
+
+namespace cb {
+DebugKnobs debug_knobs() { return DebugKnobs{g_spin_limit.load(), g_withhold.load()}; }
+}  // namespace cb
 
 extern "C" {
 
@@ -114,11 +122,28 @@ const_status_t const_csf_set_bins(const_csf_t *h, int64_t light_max_nnz, int64_t
 
 const_status_t const_csf_bin_counts(const const_csf_t *h, int64_t *n_light, int64_t *n_heavy, int64_t *n_giant,
                                     int64_t *n_items) {
-    const const_csf *c = as_csf(h);
+    const_csf *c = const_cast<const_csf *>(as_csf(h));
     if (!c) return CONST_ERR_INVALID_ARG;
+    const_status_t rc = csf_bin_totals(c);
+    if (rc != CONST_OK) return rc;
     if (n_light) *n_light = c->n_light;
     if (n_heavy) *n_heavy = c->n_heavy;
     if (n_giant) *n_giant = c->n_giant;
+    if (n_items) *n_items = c->n_items;
+    return CONST_OK;
+}
+
+const_status_t const_csf_work_lists(const const_csf_t *h, const int32_t **slice_ptr, const int32_t **light_list,
+                                    int64_t *n_light, const int32_t **items, int64_t *n_items) {
+    const_csf *c = const_cast<const_csf *>(as_csf(h));
+    if (!c) return CONST_ERR_INVALID_ARG;
+    const_status_t rc = csf_bin_totals(c);
+    if (rc != CONST_OK) return rc;
+    static_assert(sizeof(WorkItem) == 4 * sizeof(int32_t), "a work item is four int32");
+    if (slice_ptr) *slice_ptr = c->slice_ptr;
+    if (light_list) *light_list = c->light_list;
+    if (n_light) *n_light = c->n_light;
+    if (items) *items = reinterpret_cast<const int32_t *>(c->items);
     if (n_items) *n_items = c->n_items;
     return CONST_OK;
 }
@@ -203,13 +228,36 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
     if (!p || !operands || n_operands < 1 || !out_dev) return CONST_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const PlanDesc &d = p->desc;
+    // the kernels read factor rows and write results with 128-bit accesses: refuse a pointer they would fault on
+    // (checked before anything touches the device)
+    if (!aligned16(out_dev)) return CONST_ERR_INVALID_ARG;
+    for (int i = 0; i < n_operands; ++i)
+        if (operands[i].dense_dev && !aligned16(operands[i].dense_dev)) return CONST_ERR_INVALID_ARG;
     int dev = 0;
     CB_CUDA(cudaGetDevice(&dev));
-    if (!p->status_dev || p->device != dev) {
-        if (p->status_dev) return CONST_ERR_INVALID_ARG;          // a plan stays on the device of its first use
-        CB_CUDA(cudaMalloc((void **)&p->status_dev, sizeof(int32_t)));
-        CB_CUDA(cudaMemset(p->status_dev, 0, sizeof(int32_t)));
-        p->device = dev;
+    {
+        // The status word is allocated and cleared in the order of the caller's stream at the first execute,
+        // so that this call stays asynchronous; an execute on another stream waits (on the device) for the clear.
+        std::lock_guard<std::mutex> lock(p->mu);
+        if (p->status_dev && p->device != dev) return CONST_ERR_INVALID_ARG;   // a plan stays on the device of its first use
+        if (!p->status_dev) {
+            int32_t *word = nullptr;
+            cudaEvent_t ready = nullptr;
+            CB_CUDA(cudaMallocAsync((void **)&word, sizeof(int32_t), stream));
+            if (cudaMemsetAsync(word, 0, sizeof(int32_t), stream) != cudaSuccess ||
+                cudaEventCreateWithFlags(&ready, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventRecord(ready, stream) != cudaSuccess) {
+                if (ready) cudaEventDestroy(ready);
+                cudaFreeAsync(word, stream);
+                return CONST_ERR_CUDA;
+            }
+            p->status_dev = word;
+            p->status_stream = stream;
+            p->status_ready = ready;
+            p->device = dev;
+        } else if (stream != p->status_stream) {
+            CB_CUDA(cudaStreamWaitEvent(stream, p->status_ready, 0));
+        }
     }
     // bind operands by name
     const const_operand_t *x = find_operand(operands, n_operands, d.sparse_name);
@@ -269,10 +317,10 @@ const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
 const_status_t const_last_device_status(const_plan_t *h, void *stream) {
     const_plan *p = const_cast<const_plan *>(as_plan(h));
     if (!p) return CONST_ERR_INVALID_ARG;
-    CB_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-    if (!p->status_dev) return CONST_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t s = 0;
-    CB_CUDA(cudaMemcpy(&s, p->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (p->status_dev) CB_CUDA(cudaMemcpyAsync(&s, p->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CB_CUDA(cudaStreamSynchronize(st));
     return (const_status_t)s;
 }
 
@@ -288,12 +336,22 @@ void const_destroy(void *handle) {
             int prev = 0;
             cudaGetDevice(&prev);
             cudaSetDevice(p->device);
-            cudaFree(p->status_dev);
+            cudaFree(p->status_dev);               // waits for outstanding work, then releases the stream-ordered allocation
+            if (p->status_ready) cudaEventDestroy(p->status_ready);
             cudaSetDevice(prev);
         }
         p->magic = 0;
         delete p;
     }
+}
+
+const_status_t const_debug_set(int what, int64_t value) {
+    if (value < 0 || value > 0x7fffffff) return CONST_ERR_INVALID_ARG;
+    switch (what) {
+        case 0: g_spin_limit.store((int)value); return CONST_OK;
+        case 1: g_withhold.store(value != 0); return CONST_OK;
+    }
+    return CONST_ERR_INVALID_ARG;
 }
 
 const char *const_status_string(const_status_t s) {

@@ -61,9 +61,10 @@ __device__ __forceinline__ int32_t lower_bound_pos(const int32_t *__restrict__ p
 }
 
 __global__ void __launch_bounds__(kWarps * 32, 8)
-chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ light_list, Csf3 x,
+chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ bin_totals,
+                 const int32_t *__restrict__ light_list, Csf3 x,
                  const float *__restrict__ U, const float *__restrict__ V, float *__restrict__ out,
-                 int32_t *__restrict__ status) {
+                 int32_t *__restrict__ status, int wait_polls, int withhold) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t mbar_all[kWarps];
     __shared__ uint32_t tmem_base_s;
@@ -71,6 +72,7 @@ chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__
     __shared__ int32_t tile_row[kWarpsPerBlock];
     __shared__ int32_t failed;
 
+    if ((int)blockIdx.x >= work_item_count(bin_totals)) return;      // the grid is an upper bound; nothing is held yet
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const WorkItem it = items[blockIdx.x];
     const bool light = it.kind == kItemLight;
@@ -138,7 +140,7 @@ chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__
         float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
         if ((vm >> (slot_b * SL)) & 1u) u = ldg4(U + (size_t)Jslot[slot_b] * R + 4 * quarter);
         if (pending) {                                            // the MMAs of the previous flush still read the operands
-            bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+            bool done = lane == 0 ? mbar_wait(mbar, parity, wait_polls) : true;
             done = __shfl_sync(0xffffffffu, done, 0);
             parity ^= 1;
             pending = false;
@@ -173,10 +175,12 @@ chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__
             if (lane == 0) {
                 const uint64_t a_hi = smem_desc(ahi_s, 256, 128), a_lo = smem_desc(alo_s, 256, 128);
                 const uint64_t b_hi = smem_desc(bhi_s, 4 * B_QUAD, 128), b_lo = smem_desc(blo_s, 4 * B_QUAD, 128);
-                umma_tf32(d_tmem, a_hi, b_hi, kIdesc, first ? 0u : 1u);
-                umma_tf32(d_tmem, a_lo, b_hi, kIdesc, 1u);
-                umma_tf32(d_tmem, a_hi, b_lo, kIdesc, 1u);
-                umma_commit(mbar);
+                if (!withhold) {      // (test hook: nothing issued, nothing committed -> the next bounded wait runs out)
+                    umma_tf32(d_tmem, a_hi, b_hi, kIdesc, first ? 0u : 1u);
+                    umma_tf32(d_tmem, a_lo, b_hi, kIdesc, 1u);
+                    umma_tf32(d_tmem, a_hi, b_lo, kIdesc, 1u);
+                    umma_commit(mbar);
+                }
             }
             pending = true;
             first = false;
@@ -243,7 +247,7 @@ chain3_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__
         if (ok && __any_sync(0xffffffffu, cnt > 0)) flush();
     }
     if (pending) {
-        bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+        bool done = lane == 0 ? mbar_wait(mbar, parity, wait_polls) : true;
         done = __shfl_sync(0xffffffffu, done, 0);
         if (!done) ok = false;
     }
@@ -293,11 +297,13 @@ const_status_t run_ttmc3_tensor(const const_csf *X, const float *U, const float 
                                 int64_t n_rows, int32_t *status, cudaStream_t stream) {
     if (R2 != R || R3 != R) return CONST_ERR_UNSUPPORTED;
     CB_CUDA(cudaMemsetAsync(Y, 0, sizeof(float) * TILE * n_rows, stream));
-    if (X->n_items == 0) return CONST_OK;
+    if (X->nnz == 0) return CONST_OK;
     Csf3 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], static_cast<const float *>(X->vals)};
     constexpr size_t dyn = kWarpBytes * kWarps;
+    const DebugKnobs knobs = debug_knobs();
     CB_LAUNCH("chain3_tc_kernel", stream,
-              chain3_tc_kernel<<<(unsigned)X->n_items, kWarps * 32, dyn, stream>>>(X->items, X->light_list, x, U, V, Y, status));
+              chain3_tc_kernel<<<(unsigned)X->item_cap, kWarps * 32, dyn, stream>>>(X->items, X->bin_totals, X->light_list, x, U, V, Y, status,
+                                                                                 knobs.spin_limit > 0 ? knobs.spin_limit : kMbarPolls, knobs.withhold));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }

@@ -234,7 +234,8 @@ __device__ __forceinline__ void phase2(const float *__restrict__ F1, int cnt_pad
 
 template <int R2, int R3, bool HADAMARD>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-chain3_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ light_list, Csf3 x,
+chain3_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ bin_totals,
+              const int32_t *__restrict__ light_list, Csf3 x,
               const float *__restrict__ F1, const float *__restrict__ F2, float *__restrict__ out) {
     using S = Shape<R2, R3, HADAMARD>;
     extern __shared__ __align__(16) float Ts_all[];          // [warp][WINDOW * R3] parked rows
@@ -244,6 +245,7 @@ chain3_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ li
     __shared__ int32_t Hf_all[kWarpsPerBlock][S::G1];
     __shared__ float tile[S::TILE];
 
+    if ((int)blockIdx.x >= work_item_count(bin_totals)) return;      // the grid is an upper bound
     const WorkItem it = items[blockIdx.x];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool light = it.kind == kItemLight;
@@ -315,20 +317,15 @@ const_status_t launch_chain3(const const_csf *X, const float *F1, const float *F
                              cudaStream_t stream) {
     constexpr int TILE = Shape<R2, R3, HADAMARD>::TILE;
     CB_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * TILE * n_rows, stream));       // "R[*] = 0" precedes the nest
-    if (X->n_items == 0) return CONST_OK;
+    if (X->nnz == 0) return CONST_OK;
     Csf3 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], static_cast<const float *>(X->vals)};
     using S = Shape<R2, R3, HADAMARD>;
     constexpr size_t dyn = sizeof(float) * kWarpsPerBlock * S::WINDOW * R3;
-    static bool attr_set[64] = {false};                     // per template instance and device
-    int dev = 0;
-    CB_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        CB_CUDA(cudaFuncSetAttribute(chain3_kernel<R2, R3, HADAMARD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    static PerDeviceOnce attr_once;                     // per template instance
+    CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(chain3_kernel<R2, R3, HADAMARD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); }));
     CB_LAUNCH("chain3_kernel", stream,
-              chain3_kernel<R2, R3, HADAMARD><<<(unsigned)X->n_items, kWarpsPerBlock * 32, dyn, stream>>>(
-                  X->items, X->light_list, x, F1, F2, out));
+              chain3_kernel<R2, R3, HADAMARD><<<(unsigned)X->item_cap, kWarpsPerBlock * 32, dyn, stream>>>(
+                  X->items, X->bin_totals, X->light_list, x, F1, F2, out));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }

@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
                                                             const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
                                                             int shift, const uint32_t *__restrict__ digit_base,
                                                             unsigned long long *status, uint32_t *counter,
-                                                            int32_t *err, unsigned epoch) {
+                                                            int32_t *err, unsigned epoch, int spin_limit, int withhold) {
     constexpr int kBins = 1 << BITS;
     constexpr unsigned kDigitMask = kBins - 1;
     constexpr int DPT = kBins / kRsThreads;
@@ -172,7 +172,8 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     for (int q = 0; q < DPT; ++q) {
         const int d = q * kRsThreads + threadIdx.x;
         count[q] = tile_hist[d];
-        st[(size_t)tile * kBins + d] = status_word(epoch, tile == 0 ? kFlagPrefix : kFlagOwn, count[q]);
+        if (!withhold)      // (test hook: with the counts withheld, every later tile's bounded wait runs out)
+            st[(size_t)tile * kBins + d] = status_word(epoch, tile == 0 ? kFlagPrefix : kFlagOwn, count[q]);
     }
 
     // Rank inside the warp: keys with equal digits keep their order (item, lane).  The lanes holding
@@ -307,7 +308,7 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
                 unsigned long long v = *p;
                 int spins = 0;
                 while ((unsigned)(v >> 32) != tag_own && (unsigned)(v >> 32) != tag_prefix) {
-                    if (++spins > kSpinLimit) { ok = false; break; }
+                    if (++spins > spin_limit) { ok = false; break; }
                     __nanosleep(spins < 8 ? 200 : 1000);   // back off at once: polling warps must not crowd the issue slots
                     v = *p;
                 }
@@ -317,7 +318,7 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
                 p -= kBins;
                 --togo;
             }
-            if (ok) st[(size_t)tile * kBins + d] = status_word(epoch, kFlagPrefix, before + count[q]);
+            if (ok && !withhold) st[(size_t)tile * kBins + d] = status_word(epoch, kFlagPrefix, before + count[q]);
         }
         s_gbase[d] = digit_base[d] + before - excl[q];      // modulo 2^32; adding a tile-local position gives the true offset
     }
@@ -630,10 +631,10 @@ __global__ void bin_fill(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int
 // One thread per block work item of the heavy/giant range: items of giant slices find their own
 // level-1 node range (the slice is cut where the leaf offset passes q/parts of its nonzeros).
 __global__ void bin_fill_chunks(ChainPtrs c, const int32_t *__restrict__ slice_ptr, int64_t n0, int64_t heavy_max,
-                                int64_t chunk, const int32_t *__restrict__ item_off, int64_t n_hg_items,
-                                WorkItem *__restrict__ items) {
+                                int64_t chunk, const int32_t *__restrict__ item_off,
+                                const int32_t *__restrict__ totals, WorkItem *__restrict__ items) {
     int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= n_hg_items) return;
+    if (t >= totals[0]) return;                       // the grid covers the upper bound of the item count
     // slice owning item t: last s with item_off[s] <= t (slices without items share their successor's offset)
     int64_t lo = 0, hi = n0 - 1;
     while (lo < hi) {
@@ -662,7 +663,8 @@ __global__ void bin_fill_chunks(ChainPtrs c, const int32_t *__restrict__ slice_p
     items[t] = WorkItem{(int32_t)s, cut[0], cut[1], kItemChunk};
 }
 
-__global__ void bin_light_items(WorkItem *__restrict__ items, int64_t first_item, int64_t n_light) {
+__global__ void bin_light_items(WorkItem *__restrict__ items, const int32_t *__restrict__ totals) {
+    const int64_t first_item = totals[0], n_light = totals[1];
     int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int64_t groups = (n_light + kWarpsPerBlock - 1) / kWarpsPerBlock;
     if (g >= groups) return;
@@ -681,7 +683,9 @@ int bits_for(int64_t extent) {
 // is unlimited, so buffers freed by one build are reused by the next without going back to the driver.
 cudaMemPool_t library_pool(int device) {
     static cudaMemPool_t pools[64] = {nullptr};
+    static std::mutex mu;
     if (device < 0 || device >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
     if (!pools[device]) {
         cudaMemPoolProps props;
         std::memset(&props, 0, sizeof(props));
@@ -739,16 +743,13 @@ const_status_t launch_onesweep(const uint64_t *kin, uint64_t *kout, const V *vin
                                unsigned epoch, cudaStream_t stream) {
     const int64_t ntiles = (n + kRsTile - 1) / kRsTile;
     const size_t dyn = kRsTile * (sizeof(uint64_t) + sizeof(V));
-    static bool attr_set[64] = {false};    // per template instance and device
-    int dev = 0;
-    CB_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        CB_CUDA(cudaFuncSetAttribute(rs_onesweep<V, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    static PerDeviceOnce attr_once;                     // per template instance
+    CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(rs_onesweep<V, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); }));
+    const DebugKnobs knobs = debug_knobs();
     CB_LAUNCH("rs_onesweep", stream,
               rs_onesweep<V, BITS><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(
-                  kin, kout, vin, vout, n, shift, digit_base, b.tile_status, counter, status, epoch));
+                  kin, kout, vin, vout, n, shift, digit_base, b.tile_status, counter, status, epoch,
+                  knobs.spin_limit > 0 ? knobs.spin_limit : kSpinLimit, knobs.withhold));
     return CONST_OK;
 }
 
@@ -898,37 +899,62 @@ cudaError_t wait_stream(cudaStream_t stream) {
     return cudaStreamSynchronize(stream);          // something takes seconds: stop burning a core
 }
 
+// Upper bound of the number of work items for the current thresholds: a light or heavy slice gives at most
+// one item, a giant slice of z nonzeros ceil(z / chunk) <= z / chunk + 1.
+int64_t item_capacity(const const_csf *csf) {
+    return csf->n[0] + csf->nnz / std::max<int64_t>(csf->chunk, 1) + 1;
+}
+
 const_status_t csf_rebin(const_csf *csf, cudaStream_t stream) {
     const int64_t n0 = csf->n[0];
-    if (csf->light_list) { cudaFreeAsync(csf->light_list, stream); csf->light_list = nullptr; }
-    if (csf->items) { cudaFreeAsync(csf->items, stream); csf->items = nullptr; }
     csf->n_light = csf->n_heavy = csf->n_giant = csf->n_items = 0;
-    if (n0 == 0) return CONST_OK;
+    csf->totals_on_host = n0 == 0;
+    csf->bin_stream = stream;
+    if (n0 == 0) { csf->item_cap = 0; return CONST_OK; }
+    // Nothing below waits for the device: the lists are sized by their upper bounds, the fill kernels read
+    // the counts the scan left in `totals`, and so do the fused kernels later on.
+    const int64_t cap = item_capacity(csf);
+    if (cap > 0x7fffffffll) return CONST_ERR_UNSUPPORTED;
+    if (cap > csf->item_cap || !csf->items) {
+        if (csf->items) cudaFreeAsync(csf->items, stream);
+        csf->items = nullptr;
+        CB_CUDA(pool_alloc((void **)&csf->items, sizeof(WorkItem) * cap, stream));
+    }
+    csf->item_cap = cap;
+    if (!csf->light_list) CB_CUDA(pool_alloc((void **)&csf->light_list, sizeof(int32_t) * n0, stream));
     ChainPtrs c;
     c.order = csf->order;
     for (int l = 0; l < kMaxOrder; ++l) c.pos[l] = csf->pos[l];
     int32_t *item_off = csf->bin_scratch, *light_idx = csf->bin_scratch + (n0 + 1), *totals = csf->bin_scratch + 2 * (n0 + 1);
+    csf->bin_totals = totals;
     CB_LAUNCH("bin_scan", stream, bin_scan<<<1, 1024, 0, stream>>>(csf->slice_ptr, n0, csf->light_max, csf->heavy_max, csf->chunk, item_off,
                                      light_idx, totals));
-    int32_t h[4];
-    CB_CUDA(cudaMemcpyAsync(h, totals, sizeof(h), cudaMemcpyDeviceToHost, stream));
-    CB_CUDA(wait_stream(stream));
-    const int64_t hg_items = h[0];
+    CB_LAUNCH("bin_fill", stream, bin_fill<<<(unsigned)((n0 + 255) / 256), 256, 0, stream>>>(c, csf->slice_ptr, n0, csf->light_max, csf->heavy_max,
+                                                              item_off, totals + 8, csf->items, csf->light_list));
+    CB_LAUNCH("bin_fill_chunks", stream, bin_fill_chunks<<<(unsigned)((cap + 127) / 128), 128, 0, stream>>>(
+                  c, csf->slice_ptr, n0, csf->heavy_max, csf->chunk, item_off, totals, csf->items));
+    const int64_t max_groups = (n0 + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    CB_LAUNCH("bin_light_items", stream, bin_light_items<<<(unsigned)((max_groups + 255) / 256), 256, 0, stream>>>(csf->items, totals));
+    CB_CUDA(cudaGetLastError());
+    return CONST_OK;
+}
+
+// Host copies of the bin totals, for callers that ask (const_csf_bin_counts, const_csf_work_lists).
+const_status_t csf_bin_totals(const_csf *csf) {
+    if (csf->totals_on_host) return CONST_OK;
+    int32_t h[4] = {0, 0, 0, 0};
+    int prev = 0;
+    CB_CUDA(cudaGetDevice(&prev));
+    CB_CUDA(cudaSetDevice(csf->device));
+    cudaError_t e = cudaMemcpyAsync(h, csf->bin_totals, sizeof(h), cudaMemcpyDeviceToHost, csf->bin_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(csf->bin_stream);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) return CONST_ERR_CUDA;
     csf->n_light = h[1];
     csf->n_heavy = h[2];
     csf->n_giant = h[3];
-    const int64_t light_groups = (csf->n_light + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    csf->n_items = hg_items + light_groups;
-    CB_CUDA(pool_alloc((void **)&csf->items, sizeof(WorkItem) * std::max<int64_t>(csf->n_items, 1), stream));
-    CB_CUDA(pool_alloc((void **)&csf->light_list, sizeof(int32_t) * std::max<int64_t>(csf->n_light, 1), stream));
-    CB_LAUNCH("bin_fill", stream, bin_fill<<<(unsigned)((n0 + 255) / 256), 256, 0, stream>>>(c, csf->slice_ptr, n0, csf->light_max, csf->heavy_max,
-                                                              item_off, totals + 8, csf->items, csf->light_list));
-    if (hg_items > 0)
-        CB_LAUNCH("bin_fill_chunks", stream, bin_fill_chunks<<<(unsigned)((hg_items + 127) / 128), 128, 0, stream>>>(
-                      c, csf->slice_ptr, n0, csf->heavy_max, csf->chunk, item_off, hg_items, csf->items));
-    if (light_groups > 0)
-        CB_LAUNCH("bin_light_items", stream, bin_light_items<<<(unsigned)((light_groups + 255) / 256), 256, 0, stream>>>(csf->items, hg_items, csf->n_light));
-    CB_CUDA(cudaGetLastError());
+    csf->n_items = h[0] + (h[1] + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    csf->totals_on_host = true;
     return CONST_OK;
 }
 
@@ -1066,6 +1092,8 @@ const_status_t noalloc_scratch(unsigned char **out) {
     int dev = 0;
     CB_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kNaMaxDevices) return CONST_ERR_UNSUPPORTED;
+    static std::mutex mu;                                                     // two host threads may arrive first together
+    std::lock_guard<std::mutex> lock(mu);
     if (!g_noalloc_ptr[dev]) {
         void *p = nullptr;
         CB_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));                 // resolved with `dev` current

@@ -252,7 +252,9 @@ const_status_t run_network(const const_csf *U, const double *V, const const_csf 
     const size_t smem = sizeof(double) * t_doubles + sizeof(Rec) * RB + sizeof(int32_t) * (2 * FPMAX + 1);
     if (smem > 220 * 1024 || n_l > (1ll << 30) || n_m > (1ll << 30)) return CONST_ERR_WORKSPACE;
     auto kernel = network_kernel<IS, GL>;
-    CB_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // the requested size depends on n_k: raise the limit once per device to the most a block may have
+    static PerDeviceOnce attr_once;
+    CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024); }));
     Csf3d u{U->crd[0], U->pos[1], U->crd[1], U->pos[2], U->crd[2], static_cast<const double *>(U->vals), (int32_t)U->n[0]};
     Csf3d w{W->crd[0], W->pos[1], W->crd[1], W->pos[2], W->crd[2], static_cast<const double *>(W->vals), (int32_t)W->n[0]};
     const int v_vec_ok = (n_l % 2 == 0) && (reinterpret_cast<uintptr_t>(V) % 16 == 0);

@@ -155,7 +155,8 @@ __device__ __forceinline__ void phase1(const Csf4 &x, const float *__restrict__ 
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-ttmc4_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ light_list, Csf4 x,
+ttmc4_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ bin_totals,
+             const int32_t *__restrict__ light_list, Csf4 x,
              const float *__restrict__ U, const float *__restrict__ V, const float *__restrict__ W,
              float *__restrict__ out) {
     extern __shared__ __align__(16) float Qs_all[];              // [warp][WF * 64] parked Q
@@ -165,6 +166,7 @@ ttmc4_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ lig
     __shared__ int32_t Hf_all[kWarpsPerBlock][G];
     __shared__ float tile[TILE];
 
+    if ((int)blockIdx.x >= work_item_count(bin_totals)) return;      // the grid is an upper bound
     const WorkItem it = items[blockIdx.x];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool light = it.kind == kItemLight;
@@ -250,18 +252,13 @@ const_status_t run_ttmc4(const const_csf *X, const float *U, const float *V, con
                          int64_t n_rows, int32_t *, cudaStream_t stream) {
     if (rank != R) return CONST_ERR_UNSUPPORTED;
     CB_CUDA(cudaMemsetAsync(Y, 0, sizeof(float) * TILE * n_rows, stream));
-    if (X->n_items == 0) return CONST_OK;
+    if (X->nnz == 0) return CONST_OK;
     Csf4 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], X->pos[3], X->crd[3],
            static_cast<const float *>(X->vals)};
     constexpr size_t dyn = sizeof(float) * kWarpsPerBlock * WF * QROW;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    CB_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        CB_CUDA(cudaFuncSetAttribute(ttmc4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
-    CB_LAUNCH("ttmc4_kernel", stream, ttmc4_kernel<<<(unsigned)X->n_items, kWarpsPerBlock * 32, dyn, stream>>>(X->items, X->light_list, x, U, V, W, Y));
+    static PerDeviceOnce attr_once;                     // per template instance
+    CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(ttmc4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); }));
+    CB_LAUNCH("ttmc4_kernel", stream, ttmc4_kernel<<<(unsigned)X->item_cap, kWarpsPerBlock * 32, dyn, stream>>>(X->items, X->bin_totals, X->light_list, x, U, V, W, Y));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }

@@ -101,9 +101,10 @@ __device__ __forceinline__ NodeInfo load_node(const Csf4 &x, int32_t n, int32_t 
 }
 
 __global__ void __launch_bounds__(kWarps * 32, 5)
-ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *__restrict__ light_list, Csf4 x,
+ttmc4_tc_kernel(const WorkItem *__restrict__ items, const int32_t *__restrict__ bin_totals,
+                const int32_t *__restrict__ light_list, Csf4 x,
                 const float *__restrict__ U, const float *__restrict__ V, const float *__restrict__ W,
-                float *__restrict__ out, int32_t *__restrict__ status) {
+                float *__restrict__ out, int32_t *__restrict__ status, int wait_polls, int withhold) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t mbar_all[kWarps];
     __shared__ uint32_t tmem_base_s;
@@ -111,6 +112,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
     __shared__ int32_t acc_used[kWarps];         // the warp issued at least one MMA
     __shared__ int32_t failed;
 
+    if ((int)blockIdx.x >= work_item_count(bin_totals)) return;      // the grid is an upper bound; nothing is held yet
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const WorkItem it = items[blockIdx.x];
     const bool light = it.kind == kItemLight;
@@ -182,7 +184,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
             u1 = ldg4(up + 4);
         }
         if (pending) {                                            // the MMAs of the previous flush still read the operands
-            bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+            bool done = lane == 0 ? mbar_wait(mbar, parity, wait_polls) : true;
             done = __shfl_sync(0xffffffffu, done, 0);
             parity ^= 1;
             pending = false;
@@ -217,7 +219,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
             __syncwarp();
             if (lane == 0) {
 #pragma unroll
-                for (int kg = 0; kg < KG; ++kg) {
+                for (int kg = 0; kg < KG && !withhold; ++kg) {   // (test hook: nothing issued, nothing committed)
                     const uint64_t a_hi = smem_desc(ahi_s + kg * 2048, 1024, 128), a_lo = smem_desc(alo_s + kg * 2048, 1024, 128);
                     const uint64_t b_hi = smem_desc(bhi_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
                     const uint64_t b_lo = smem_desc(blo_s + kg * (8 * B_QUAD), 4 * B_QUAD, 128);
@@ -225,7 +227,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
                     umma_tf32(d_tmem, a_lo, b_hi, kIdesc, 1u);
                     umma_tf32(d_tmem, a_hi, b_lo, kIdesc, 1u);
                 }
-                umma_commit(mbar);
+                if (!withhold) umma_commit(mbar);               // withheld: the next bounded wait runs out
                 acc_used[warp] = 1;
             }
             pending = true;
@@ -319,7 +321,7 @@ ttmc4_tc_kernel(const WorkItem *__restrict__ items, int n_items, const int32_t *
         if (ok && __any_sync(0xffffffffu, cnt > 0)) flush();
     }
     if (pending) {
-        bool done = lane == 0 ? mbar_wait(mbar, parity) : true;
+        bool done = lane == 0 ? mbar_wait(mbar, parity, wait_polls) : true;
         done = __shfl_sync(0xffffffffu, done, 0);
         if (!done) ok = false;
     }
@@ -388,20 +390,17 @@ const_status_t run_ttmc4_tensor(const const_csf *X, const float *U, const float 
                                 int64_t n_rows, int32_t *status, cudaStream_t stream) {
     if (rank != R) return CONST_ERR_UNSUPPORTED;
     CB_CUDA(cudaMemsetAsync(Y, 0, sizeof(float) * TILE * n_rows, stream));
-    if (X->n_items == 0) return CONST_OK;
+    if (X->nnz == 0) return CONST_OK;
     Csf4 x{X->crd[0], X->pos[1], X->crd[1], X->pos[2], X->crd[2], X->pos[3], X->crd[3],
            static_cast<const float *>(X->vals)};
     constexpr size_t dyn = kWarpBytes * kWarps;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    CB_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        CB_CUDA(cudaFuncSetAttribute(ttmc4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
-    const unsigned grid = (unsigned)X->n_items;
+    static PerDeviceOnce attr_once;                     // per template instance
+    CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(ttmc4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); }));
+    const unsigned grid = (unsigned)X->item_cap;
+    const DebugKnobs knobs = debug_knobs();
     CB_LAUNCH("ttmc4_tc_kernel", stream,
-              ttmc4_tc_kernel<<<grid, kWarps * 32, dyn, stream>>>(X->items, (int)X->n_items, X->light_list, x, U, V, W, Y, status));
+              ttmc4_tc_kernel<<<grid, kWarps * 32, dyn, stream>>>(X->items, X->bin_totals, X->light_list, x, U, V, W, Y, status,
+                                                               knobs.spin_limit > 0 ? knobs.spin_limit : kMbarPolls, knobs.withhold));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
 }

@@ -48,8 +48,9 @@ __device__ __forceinline__ void umma_commit(uint32_t mbar) {
 }
 
 // true when the phase with the given parity has completed; gives up after a bounded number of polls
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
-    for (int it = 0; it < (1 << 20); ++it) {
+constexpr int kMbarPolls = 1 << 20;
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, int polls = kMbarPolls) {
+    for (int it = 0; it < polls; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"

@@ -5,6 +5,7 @@ import torch
 import paper_2401_04836_b200 as cb
 from oracle import contract as oc
 from oracle import csf as ocsf
+from oracle import workload as ow
 
 TOL = {np.dtype(np.float32): 1e-5, np.dtype(np.float64): 1e-12}    # |gpu - S| <= TOL * A per element
 
@@ -59,24 +60,7 @@ def run_workload(w, bins=None, handles=None, tensor_stage=None):
 
 def oracle(w, rows=None):
     """(S, A) of the workload's expression; rows = only these output rows (others are returned as zeros)."""
-    from workloads import row_sample
-    fam = w.family
-    if fam == "network":
-        U, W = w.sparse["U"], w.sparse["W"]
-        if rows is not None:
-            U = row_sample(U, rows)
-        return oc.network(U.coords, U.vals, w.dense["V"], W.coords, W.vals, w.extents["i"], w.extents["k"],
-                          w.extents["m"])
-    X = w.sparse["X"]
-    if rows is not None:
-        X = row_sample(X, rows)
-    if fam == "ttmc3":
-        return oc.ttmc3(X.coords, X.vals, w.dense["U"], w.dense["V"], X.dims[0])
-    if fam == "ttmc4":
-        return oc.ttmc4(X.coords, X.vals, w.dense["U"], w.dense["V"], w.dense["W"], X.dims[0])
-    if fam == "mttkrp":
-        return oc.mttkrp3(X.coords, X.vals, w.dense["B"], w.dense["C"], X.dims[0])
-    raise ValueError(fam)
+    return ow.evaluate(w, rows)
 
 
 def assert_close(out, S, A, dtype, rows=None):

@@ -37,3 +37,35 @@ def test_status_strings_and_null_handling():
     assert lib.const_csf_build(3, None, 0, None, None, 0, None, None, ctypes.byref(out)) == 1
     assert lib.const_execute(None, None, 0, None, None) == 1
     assert lib.const_csf_level(None, 0, None, None, None) == 1
+
+
+def test_execute_refuses_misaligned_pointers_before_touching_the_device():
+    """Dense operands and the output are read and written with 128-bit accesses: a pointer that is not
+    16-byte aligned is refused with CONST_ERR_INVALID_ARG before any device call."""
+    import torch
+    from workloads import make_config
+    w = make_config(1)
+    plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, cb.F32)
+    lib = ctypes.CDLL(cb.library_path())                      # its own function objects: the binding's prototypes stay as they are
+
+    class Operand(ctypes.Structure):
+        _fields_ = [("name", ctypes.c_char_p), ("csf", ctypes.c_void_p), ("dense_dev", ctypes.c_void_p)]
+
+    fake_csf = ctypes.create_string_buffer(1024)              # zeroed: not a CSF handle (wrong magic)
+    base = 0x7f0000001000                                     # never dereferenced on the paths below
+
+    def run(u_ptr, v_ptr, out_ptr):
+        ops = (Operand * 3)(Operand(b"X", ctypes.addressof(fake_csf), None), Operand(b"U", None, u_ptr),
+                            Operand(b"V", None, v_ptr))
+        return lib.const_execute(ctypes.c_void_p(plan.ptr), ctypes.cast(ops, ctypes.c_void_p), 3,
+                                 ctypes.c_void_p(out_ptr), None)
+
+    lib.const_execute.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+    assert run(base + 4, base, base) == 1                     # factor row base off by one float
+    assert run(base, base + 8, base) == 1
+    assert run(base, base, base + 4) == 1                     # output
+    aligned = run(base, base, base)
+    if not torch.cuda.is_available():
+        assert aligned == 7                                   # got past the alignment check to the first device call
+    else:
+        assert aligned == 1                                   # the fake CSF handle is refused; nothing was launched

@@ -1,13 +1,15 @@
 """The five benchmark configurations at full size, in the launch configuration bench.py times.
 
-The oracle cannot sort 10^8 nonzeros or evaluate 10^10 terms in seconds, so every check is either a
-property that holds at any size or an exact comparison on sampled slices:
-  * CSF: level sizes against distinct-prefix counts computed on the host; pos/crd invariants over the
-    whole arrays; for sampled root slices (the largest one included) every array segment bit-exact
-    against the CSF oracle built from that slice's nonzeros alone;
-  * contraction: sampled output rows element by element against the fp64 oracle run on the nonzeros
-    of those rows (|gpu - S| <= tol * sum|terms|); every other row finite.
+  * CSF: the oracle cannot sort 10^8 nonzeros in seconds, so the arrays are checked by properties
+    that hold at any size (level sizes against distinct-prefix counts computed on the host; pos/crd
+    invariants over the whole arrays) and, for sampled root slices (the largest and the smallest
+    included), every array segment bit-exact against the CSF oracle built from that slice alone;
+  * contraction: EVERY output row, element by element, against the fp64 oracle evaluated on the whole
+    tensor (|gpu - S| <= tol * sum|terms|, and exactly 0 where no term exists).  The oracle result of a
+    configuration is computed once and shared by the parametrisations that use it.
 """
+import functools
+
 import numpy as np
 import pytest
 import torch
@@ -74,10 +76,21 @@ def _check_csf(h, op, mode_order, rows):
         assert vals[lo:hi].cpu().numpy().tobytes() == ovals.tobytes(), f"values of slice {r}"
 
 
+@functools.lru_cache(maxsize=None)
+def _workload(config_id):
+    return make_config(config_id)
+
+
+@functools.lru_cache(maxsize=None)
+def _oracle_all_rows(config_id):
+    """(S, A) over every output row: tens of seconds of host time per configuration."""
+    return oracle(_workload(config_id))
+
+
 @pytest.mark.parametrize("config_id,tensor_stage", [(2, None), (2, True), (3, False), (3, True), (4, None), (5, None)])
 def test_full_size_config(config_id, tensor_stage):
     rng = np.random.default_rng(100 + config_id)
-    w = make_config(config_id)
+    w = _workload(config_id)
     dtype = cb.F32 if w.dtype == np.float32 else cb.F64
     handles = {}
     for name, op in w.sparse.items():
@@ -95,11 +108,13 @@ def test_full_size_config(config_id, tensor_stage):
     cb.const_execute(plan, operands, out)
     assert cb.const_last_device_status(plan) == 0
     out = out.cpu().numpy()
-    assert np.all(np.isfinite(out))
+    # the default thresholds put slices of this tensor into every bin the family uses, and every row is compared
     first = w.sparse["U" if w.family == "network" else "X"]
-    rows = _sample_rows(first, 0, 24 if config_id != 5 else 6, rng)
-    S, A = oracle(w, rows)
-    assert_close(out, S, A, w.dtype, rows=rows)
+    if w.family != "network":
+        counts = cb.const_csf_bin_counts(handles["X"])
+        assert counts["light"] > 0 and counts["heavy"] > 0 and counts["giant"] > 0, counts
+    S, A = _oracle_all_rows(config_id)
+    assert_close(out, S, A, w.dtype)
     # rows whose slice is empty stay exactly zero
     empty = np.setdiff1d(np.arange(first.dims[0]), first.coords[0])
     assert np.all(out[empty] == 0)
