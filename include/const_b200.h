@@ -283,6 +283,26 @@ const_status_t const_profile_enable(int on);
 const_status_t const_profile_read(char *names, int64_t names_bytes, int64_t *launches, double *total_ms,
                                   int max_kernels, int *n_kernels);
 
+/*
+ * Micro-benchmarks of the machine limits the fused kernels are rated against (the paper has no counterpart;
+ * its measurements are single-threaded CPU times).  Each kind launches one warm-up and then `repeats`
+ * back-to-back launches on `stream`, timed with two CUDA events, waits for them, and returns the mean
+ * milliseconds per launch and the work one launch does:
+ *   CONST_BENCH_FP32_FMA / CONST_BENCH_FP64_FMA   register-only fused multiply-adds on every SM; work in flop;
+ *   CONST_BENCH_TF32_MMA     tcgen05.mma kind::tf32, M 128 x N 256 x K 8, operands in shared memory, accumulator
+ *                            in tensor memory, one block per SM; work in flop;
+ *   CONST_BENCH_ROW_GATHER   rows_dev[n] (device, int32 row numbers, e.g. a leaf-level crd array) are gathered
+ *                            from a table of table_rows x rank floats (rank 8, 16 or 32) with 128-bit loads, rank / 4
+ *                            lanes per row, four rows in flight per lane; work in bytes of rows read.
+ * rows_dev, n, table_rows and rank are ignored by the first three kinds.  The call allocates its table and a
+ * status word stream-ordered and frees them before it returns.  CONST_ERR_TIMEOUT if the bounded wait for the
+ * tensor pipe gave up.
+ */
+typedef enum { CONST_BENCH_FP32_FMA = 0, CONST_BENCH_FP64_FMA = 1, CONST_BENCH_TF32_MMA = 2,
+               CONST_BENCH_ROW_GATHER = 3 } const_microbench_kind_t;
+const_status_t const_microbench(int kind, const int32_t *rows_dev, int64_t n, int64_t table_rows, int rank, int repeats,
+                                void *stream, double *ms_per_launch, double *work_per_launch);
+
 #ifdef __cplusplus
 }
 #endif

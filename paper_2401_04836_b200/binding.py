@@ -63,6 +63,8 @@ def load_library():
     lib.const_csf_bin_counts.argtypes = [vp, pp(i64), pp(i64), pp(i64), pp(i64)]
     lib.const_csf_work_lists.argtypes = [vp, pp(vp), pp(vp), pp(i64), pp(vp), pp(i64)]
     lib.const_csf_work_lists.restype = i32
+    lib.const_microbench.argtypes = [i32, vp, i64, i64, i32, i32, vp, pp(ctypes.c_double), pp(ctypes.c_double)]
+    lib.const_microbench.restype = i32
     lib.const_debug_set.argtypes = [i32, i64]
     lib.const_debug_set.restype = i32
     lib.const_plan_create.argtypes = [ctypes.c_char_p, pp(ctypes.c_char_p), i32, pp(ctypes.c_char_p),
@@ -256,6 +258,18 @@ def const_csf_work_lists(csf: CsfHandle):
     return (_dev_to_torch(sp.value, n0.value + 1 if n0.value else 0, torch.int32),
             _dev_to_torch(ll.value, n_light.value, torch.int32),
             _dev_to_torch(it.value, 4 * n_items.value, torch.int32).reshape(-1, 4))
+
+
+BENCH_FP32_FMA, BENCH_FP64_FMA, BENCH_TF32_MMA, BENCH_ROW_GATHER = 0, 1, 2, 3
+
+
+def const_microbench(kind: int, rows=None, table_rows: int = 0, rank: int = 0, repeats: int = 5, stream=None):
+    """Machine-limit micro-benchmark (see the header); returns (milliseconds per launch, work per launch)."""
+    ms, work = ctypes.c_double(), ctypes.c_double()
+    ptr, n = (None, 0) if rows is None else (ctypes.c_void_p(rows.data_ptr()), int(rows.numel()))
+    _check(load_library().const_microbench(int(kind), ptr, n, int(table_rows), int(rank), int(repeats),
+                                           _stream_ptr(stream), ctypes.byref(ms), ctypes.byref(work)), "const_microbench")
+    return ms.value, work.value
 
 
 def const_debug_set(what: int, value: int) -> None:
