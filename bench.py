@@ -350,7 +350,7 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
     ms_per_step, total_flops = aggregate_over_ranks(ms_per_step, flops, dist, "cuda")
 
     nnz_total = sum(op.nnz for op in w.sparse.values())
-    fits_l2 = step_bytes < 126e6
+    fits_l2 = exec_bytes < 126e6                 # what const_execute touches stays resident in the 126 MB L2
     flushed = None
     if fits_l2 and rank == 0:
         # the working set fits the 126 MB L2: also time the steps with L2 flushed before each of them

@@ -172,7 +172,9 @@ const_status_t const_csf_work_lists(const const_csf_t *csf, const int32_t **slic
  * modes fusion removes (3.2.5).  The tree must also compute `expression` (same inputs, same result
  * indices, an index is summed in exactly one contraction).
  *
- * Kernel families (-> CONST_ERR_UNSUPPORTED otherwise):
+ * Kernel families (hand-written fused kernels; a schedule that matches none of them runs on the generic
+ * executor described below, and CONST_ERR_UNSUPPORTED remains for schedules beyond its fixed capacities:
+ * more than 12 contractions, 16 indices, 6 CSF operands, a dense tensor of 2^31 elements or more):
  *   chain   one CSF tensor of order 3 or 4 contracted leaf level first with one dense factor per
  *           non-root level; the result is indexed by the root level followed by the rank indices in
  *           level order (TTMc), or by one rank index shared by all factors (MTTKRP).  Ranks must be
@@ -181,6 +183,17 @@ const_status_t const_csf_work_lists(const const_csf_t *csf, const int32_t **slic
  *   network T[i,k,l] = U[i,j,k] * V[j,l]; Z[i,m] = T[i,k,l] * W[k,l,m] with V dense, U in CSF with
  *           levels (i,k,j) and W in CSF with levels (l,m,k), loop orders i,k,j,l and i,l,m,k: both
  *           contractions then gather along a fibre; fused over i only (T reduced to order 2).  CONST_F64.
+ *   tree    the generic executor (Sec. 4.2: it walks the loop tree that Algorithm 1 prints as forall / where
+ *           constructs).  Any checked schedule, any number of CSF operands, fp32 or fp64: e.g. the running
+ *           example R_ijk = A_ipq B_jpr C_kqr D_jkr with X and Y as 2-D workspaces inside the fused r, j
+ *           loops (Fig. 5), order-4 MTTKRP, TTMc at other ranks, the network with U stored (i,j,k) and W
+ *           (k,l,m), or a network multiplied by a sparse 0/1 map (Sec. 5.1, Eq. 2).  The outermost loop is
+ *           spread over thread blocks; a forall walks the nodes of a CSF operand where skipping the other
+ *           coordinates cannot change the result, else the dense range of its index, and looks the other CSF
+ *           operands up; intermediates are dense workspaces over the indices fusion left them (Sec. 2.2),
+ *           cleared at every iteration of the innermost forall shared by producer and consumer.  A producer
+ *           and its consumer are fused under a forall only if the intermediate carries that index.  Slower
+ *           than the families above; results are accumulated with atomic adds.
  */
 const_status_t const_plan_create(const char *expression, const char *const *tree, int n_contractions,
                                  const char *const *sparse_names, const int *const *mode_orders, int n_sparse,
@@ -199,7 +212,7 @@ const_status_t const_schedule_check(const char *expression, const char *const *t
                                     int *reduced_orders);
 
 /* Facts about a checked plan, for tests: reduced order of the intermediate produced by contraction
- * c (0 for the last contraction), and the family ("ttmc3", "ttmc4", "mttkrp3", "network"). */
+ * c (0 for the last contraction), and the family ("ttmc3", "ttmc4", "mttkrp3", "network", "tree"). */
 const_status_t const_plan_reduced_order(const const_plan_t *plan, int contraction, int *order);
 const char *const_plan_family(const const_plan_t *plan);
 
@@ -247,6 +260,14 @@ const_status_t const_schedule_cin(const char *expression, const char *const *tre
  * const_execute.  A device-side wait that runs out is reported through const_last_device_status.
  */
 const_status_t const_plan_set_tensor_stage(const_plan_t *plan, int enable);
+
+/*
+ * enable != 0: const_execute runs this plan on the generic executor (family "tree" of const_plan_create)
+ * although a hand-written family matches it; enable == 0: back to the family.  CONST_ERR_UNSUPPORTED when
+ * the schedule exceeds the generic executor's capacities (enable != 0) or when the plan has no other
+ * kernel (enable == 0).  Host-only call.
+ */
+const_status_t const_plan_set_generic_executor(const_plan_t *plan, int enable);
 
 /* Synchronise `stream` and return the device-side status word of the plan's last executions
  * (CONST_OK, or the first error a kernel recorded, e.g. CONST_ERR_TIMEOUT). */

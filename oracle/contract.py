@@ -195,3 +195,34 @@ def nary_direct(expression: str, operands: Dict[str, Union[np.ndarray, SparseArg
 
     rec(0, {}, 1.0)
     return S, A
+
+
+def nary_einsum(expression: str, operands: Dict[str, Union[np.ndarray, SparseArg]],
+                extents: Dict[str, int]) -> Tuple[np.ndarray, np.ndarray]:
+    """The same definition as `nary_direct` for inputs a Python loop nest cannot finish: every sparse
+    operand is written out as a dense array (zeros where nothing is stored) and the sum over all index
+    values of the product of the operands (Sec. 2.1, "Tensor networks") is taken by numpy.einsum in double
+    precision, once on the values (S) and once on their absolute values (A = sum of |terms|, since the
+    absolute value of a product is the product of the absolute values).  The index space must be small
+    enough to enumerate (product of all extents up to ~1e8)."""
+    (out_name, out_idx), refs = _parse(expression)
+    letters = {}
+    for _, idx in refs + [(out_name, out_idx)]:
+        for i in idx:
+            letters.setdefault(i, chr(ord("a") + len(letters)))
+    dense = []
+    for name, idx in refs:
+        op = operands[name]
+        if isinstance(op, np.ndarray):
+            arr = np.asarray(op, dtype=np.float64)
+        else:
+            coords, vals = op
+            arr = np.zeros([extents[i] for i in idx], dtype=np.float64)
+            arr[tuple(np.asarray(c, dtype=np.int64) for c in coords)] = np.asarray(vals, dtype=np.float64)
+        if arr.shape != tuple(extents[i] for i in idx):
+            raise ValueError(f"operand {name} has shape {arr.shape}, expected {[extents[i] for i in idx]}")
+        dense.append(arr)
+    spec = ",".join("".join(letters[i] for i in idx) for _, idx in refs) + "->" + "".join(letters[i] for i in out_idx)
+    S = np.einsum(spec, *dense, optimize=False)
+    A = np.einsum(spec, *[np.abs(a) for a in dense], optimize=False)
+    return np.ascontiguousarray(S), np.ascontiguousarray(A)

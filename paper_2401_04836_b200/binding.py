@@ -82,6 +82,8 @@ def load_library():
     lib.const_last_device_status.argtypes = [vp, vp]
     lib.const_plan_set_tensor_stage.argtypes = [vp, i32]
     lib.const_plan_set_tensor_stage.restype = i32
+    lib.const_plan_set_generic_executor.argtypes = [vp, i32]
+    lib.const_plan_set_generic_executor.restype = i32
     lib.const_destroy.argtypes = [vp]
     lib.const_destroy.restype = None
     lib.const_profile_enable.argtypes = [i32]
@@ -361,6 +363,10 @@ def const_execute(plan: PlanHandle, operands: Dict[str, Union[CsfHandle, "object
 
 def const_plan_set_tensor_stage(plan: PlanHandle, enable: bool) -> None:
     _check(load_library().const_plan_set_tensor_stage(plan.ptr, 1 if enable else 0), "const_plan_set_tensor_stage")
+
+
+def const_plan_set_generic_executor(plan: PlanHandle, enable: bool) -> None:
+    _check(load_library().const_plan_set_generic_executor(plan.ptr, 1 if enable else 0), "const_plan_set_generic_executor")
 
 
 def const_last_device_status(plan: PlanHandle, stream=None) -> int:

@@ -8,8 +8,8 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libconst_b200.so")
-SOURCES = ["api.cu", "plan.cpp", "cin.cpp", "csf_build.cu", "chain_kernels.cu", "ttmc4_kernel.cu", "ttmc4_tc_kernel.cu", "chain3_tc_kernel.cu", "network_kernels.cu", "profile.cu", "microbench.cu"]
-HEADERS = ["common.cuh", "umma.cuh", "plan.h", os.path.join("..", "..", "include", "const_b200.h")]
+SOURCES = ["api.cu", "plan.cpp", "loop_tree.cpp", "csf_build.cu", "chain_kernels.cu", "ttmc4_kernel.cu", "ttmc4_tc_kernel.cu", "chain3_tc_kernel.cu", "network_kernels.cu", "profile.cu", "microbench.cu", "tree_plan.cpp", "tree_kernel.cu"]
+HEADERS = ["common.cuh", "umma.cuh", "plan.h", "loop_tree.h", "tree_exec.h", os.path.join("..", "..", "include", "const_b200.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 

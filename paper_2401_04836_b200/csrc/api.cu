@@ -159,7 +159,16 @@ const_status_t const_plan_create(const char *expression, const char *const *tree
     const_status_t rc = parse_plan(expression, tree, n_contractions, sparse_names, mode_orders, n_sparse, loop_orders,
                                    extents, n_indices, dtype, plan->desc);
     if (rc == CONST_OK) rc = check_plan(plan->desc);
-    if (rc == CONST_OK) rc = match_plan(plan->desc);
+    if (rc == CONST_OK) {
+        // every checked schedule is compiled for the generic executor; a hand-written family, where one
+        // matches, takes precedence at execute time
+        plan->tree_ok = tree::compile(plan->desc, plan->tree);
+        rc = match_plan(plan->desc);
+        if (rc == CONST_ERR_UNSUPPORTED && plan->tree_ok) {
+            plan->desc.family = Family::Tree;
+            rc = CONST_OK;
+        }
+    }
     if (rc != CONST_OK) {
         delete plan;
         return rc;
@@ -218,6 +227,7 @@ const char *const_plan_family(const const_plan_t *h) {
         case Family::Ttmc4: return "ttmc4";
         case Family::Mttkrp3: return "mttkrp3";
         case Family::Network: return "network";
+        case Family::Tree: return "tree";
         default: return "";
     }
 }
@@ -258,6 +268,24 @@ const_status_t const_execute(const_plan_t *h, const const_operand_t *operands, i
         } else if (stream != p->status_stream) {
             CB_CUDA(cudaStreamWaitEvent(stream, p->status_ready, 0));
         }
+    }
+    if (d.family == Family::Tree || p->use_tree) {
+        const tree::Compiled &cp = p->tree;
+        const const_csf *sparse[tree::kMaxSparse] = {nullptr};
+        void *global_in[tree::kMaxDense] = {nullptr};
+        for (size_t s = 0; s < cp.sparse_names.size(); ++s) {
+            const const_operand_t *o = find_operand(operands, n_operands, cp.sparse_names[s]);
+            if (!o || !o->csf || o->dense_dev) return CONST_ERR_INVALID_ARG;
+            sparse[s] = as_csf(o->csf);
+            if (!csf_matches(sparse[s], d, cp.sparse_names[s], d.dtype)) return CONST_ERR_INVALID_ARG;
+        }
+        for (size_t g = 0; g < cp.global_names.size(); ++g) {
+            if (cp.global_is_workspace[g] || (int)g == cp.result_slot) continue;
+            const const_operand_t *o = find_operand(operands, n_operands, cp.global_names[g]);
+            if (!o || !o->dense_dev || o->csf) return CONST_ERR_INVALID_ARG;
+            global_in[g] = const_cast<void *>(o->dense_dev);
+        }
+        return run_tree(cp, d.dtype, sparse, global_in, out_dev, stream);
     }
     // bind operands by name
     const const_operand_t *x = find_operand(operands, n_operands, d.sparse_name);
@@ -311,6 +339,15 @@ const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
                            (p->desc.family == Family::Ttmc3 && p->desc.ranks[0] == 16 && p->desc.ranks[1] == 16);
     if (enable && !has_stage) return CONST_ERR_UNSUPPORTED;
     p->tensor_stage = enable ? 1 : 0;
+    return CONST_OK;
+}
+
+const_status_t const_plan_set_generic_executor(const_plan_t *h, int enable) {
+    const_plan *p = const_cast<const_plan *>(as_plan(h));
+    if (!p) return CONST_ERR_INVALID_ARG;
+    if (enable && !p->tree_ok) return CONST_ERR_UNSUPPORTED;
+    if (!enable && p->desc.family == Family::Tree) return CONST_ERR_UNSUPPORTED;   // nothing else can run this plan
+    p->use_tree = enable ? 1 : 0;
     return CONST_OK;
 }
 

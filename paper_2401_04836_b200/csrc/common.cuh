@@ -8,6 +8,7 @@
 
 #include "../../include/const_b200.h"
 #include "plan.h"
+#include "tree_exec.h"
 
 namespace cb {
 
@@ -73,6 +74,9 @@ struct const_plan {
     cudaStream_t status_stream = nullptr;   // stream that allocated and cleared it
     cudaEvent_t status_ready = nullptr;     // recorded behind the clear: other streams wait for it
     int tensor_stage = 0;              // run the dense per-slice stage on the tensor cores where a kernel has one
+    cb::tree::Compiled tree;           // programs of the generic executor (compiled for every plan it can run)
+    bool tree_ok = false;
+    int use_tree = 0;                  // run the generic executor although a hand-written family matches
     int device = -1;
     std::mutex mu;                     // first-use set-up of the status word
 };
@@ -157,5 +161,9 @@ const_status_t run_ttmc3_tensor(const const_csf *X, const float *U, const float 
 const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z,
                            int64_t n_i, int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m,
                            int32_t *status, cudaStream_t stream);
+
+// tree_kernel.cu: the generic executor; sparse[slot] and global_in[slot] follow cp.sparse_names / cp.global_names
+const_status_t run_tree(const tree::Compiled &cp, const_dtype_t dtype, const const_csf *const *sparse,
+                        void *const *global_in, void *out_dev, cudaStream_t stream);
 
 }  // namespace cb

@@ -19,7 +19,7 @@ struct Contraction {
     std::string loops;        // outermost first
 };
 
-enum class Family { None, Ttmc3, Ttmc4, Mttkrp3, Network };
+enum class Family { None, Ttmc3, Ttmc4, Mttkrp3, Network, Tree };
 
 struct PlanDesc {
     TensorRef result;
@@ -48,6 +48,6 @@ const_status_t parse_plan(const char *expression, const char *const *tree, int n
                           const_dtype_t dtype, PlanDesc &out);
 const_status_t check_plan(PlanDesc &p);     // Sec. 3.2 constraints -> CONST_ERR_ILLEGAL_SCHEDULE
 const_status_t match_plan(PlanDesc &p);     // kernel family      -> CONST_ERR_UNSUPPORTED
-std::string schedule_cin(const PlanDesc &p); // cin.cpp: concrete index notation of the schedule (Algorithm 1)
+std::string schedule_cin(const PlanDesc &p); // loop_tree.cpp: concrete index notation of the schedule (Algorithm 1)
 
 }  // namespace cb

@@ -1,0 +1,101 @@
+// Generic executor for loop trees (any legal schedule): the compiled form of a schedule that the
+// interpreter kernel of tree_kernel.cu walks.  One Program per top-level entry of the loop tree.
+//
+// Execution model.  The outermost forall of an entry is spread over thread blocks.  Below it, a forall
+// whose body holds several assignments ("uniform loop") is run by all threads of the block in lockstep,
+// with a block barrier after every entry of its body; a forall chain that leads to a single assignment
+// ("private loops") is run in parallel: its first loop is dealt to the warps, its second to the lanes,
+// deeper ones run sequentially in each thread.  A loop walks the children of one CSF operand (its driver)
+// when one qualifies, otherwise the dense range of its index; the other CSF operands that carry the index
+// are located by binary search and an assignment is skipped where one of its operands has no such node.
+// Intermediates are dense workspaces over the indices fusion left them: private to a block when producer
+// and consumer share a forall (cleared at every iteration of the innermost shared one), global otherwise.
+// All accumulation is by atomic adds, so results can differ in the last bits from run to run.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "plan.h"
+
+namespace cb {
+namespace tree {
+
+constexpr int kMaxIdx = 16, kMaxLoops = 24, kMaxStmts = 12, kMaxSparse = 6, kMaxDense = 20, kMaxInstr = 96;
+constexpr int kMaxRefIdx = 6, kMaxPriv = 6, kMaxFollow = 3, kMaxLevels = 4;
+constexpr int kThreads = 256;
+
+enum RefKind : int8_t { kRefSparse = 0, kRefGlobal = 1, kRefPrivate = 2 };
+
+struct Ref {                       // one tensor reference of an assignment
+    int8_t kind;                   // RefKind
+    int8_t slot;                   // sparse slot, global pointer slot, or private workspace id
+    int8_t n;                      // indices that address it (global / private)
+    int8_t idx[kMaxRefIdx];        // index ids
+    int32_t stride[kMaxRefIdx];    // elements
+};
+
+struct Loop {
+    int8_t index;                  // index id
+    int8_t driver;                 // sparse slot whose level `level` the loop walks; -1: dense range [0, extent)
+    int8_t level;
+    int8_t n_follow;
+    int8_t follow[kMaxFollow];     // sparse slots located at the loop's coordinate ...
+    int8_t flevel[kMaxFollow];     // ... and the level of each that carries this index
+    int32_t extent;
+};
+
+struct Stmt {
+    int8_t n_priv;                 // private loops, outermost first
+    int8_t priv[kMaxPriv];         // loop ids
+    int8_t n_sparse;
+    int8_t sparse[2];              // sparse slots it reads
+    Ref out, lhs, rhs;
+};
+
+enum Op : int8_t { kOpLoopBegin = 0, kOpLoopEnd = 1, kOpZero = 2, kOpStmt = 3 };
+struct Instr { int8_t op; int8_t arg; int16_t jump; };
+
+struct Workspace { int64_t offset, size; };      // block-private: elements, offset inside the block's scratch
+
+struct Program {
+    int32_t n_instr;
+    int32_t root_loop;             // loop spread over the blocks, -1: the entry is a bare assignment
+    int64_t block_scratch;         // elements of private workspace per block
+    Instr instr[kMaxInstr];
+    Loop loops[kMaxLoops];
+    Stmt stmts[kMaxStmts];
+    Workspace ws[kMaxStmts];
+};
+
+struct SparsePtrs {
+    const int32_t *pos[kMaxLevels];
+    const int32_t *crd[kMaxLevels];
+    const void *vals;
+    int32_t n0, order;
+};
+
+struct Bindings {
+    SparsePtrs sp[kMaxSparse];
+    void *global[kMaxDense];       // dense inputs, the result, global workspaces
+    void *scratch;                 // private workspaces: block b owns [b * block_scratch, (b + 1) * block_scratch)
+};
+
+// What const_execute needs besides the programs.
+struct Compiled {
+    std::vector<Program> programs;
+    std::vector<std::string> sparse_names;                 // slot -> input name
+    std::vector<std::string> global_names;                 // slot -> input name, result name, or "" for a workspace
+    std::vector<int64_t> global_elems;                     // slot -> elements (workspaces and the result; 0 for inputs)
+    std::vector<bool> global_is_workspace;
+    int result_slot = -1;
+    std::vector<int> root_driver;                          // per program: sparse slot driving the root loop or -1
+    std::vector<int64_t> root_extent;                      // per program: extent of the root index (dense root loop)
+    std::string error;
+};
+
+// Compiles a parsed and checked schedule.  False (with `error` set) when it exceeds the fixed capacities.
+bool compile(const PlanDesc &desc, Compiled &out);
+
+}  // namespace tree
+}  // namespace cb

@@ -266,3 +266,48 @@ def test_rejects_out_of_range_coordinates():
         oc.ttmc3([np.array([0]), np.array([9]), np.array([0])], np.array([1.0]), np.ones((3, 2)), np.ones((3, 2)), 2)
     with pytest.raises(ValueError):
         oc.ttmc3([np.array([5]), np.array([0]), np.array([0])], np.array([1.0]), np.ones((3, 2)), np.ones((3, 2)), 2)
+
+
+def test_einsum_evaluator_agrees_with_the_loop_nest_evaluator():
+    """`nary_einsum` (densify + numpy.einsum) against `nary_direct` (Python loops over stored nonzeros) on the
+    running example, an order-4 MTTKRP and a network times a sparse 0/1 map; and a closed form: with every stored
+    value 1 and dense factors of ones, an output element counts the index combinations that reach it."""
+    rng = np.random.default_rng(16)
+    n = 3
+    ops = _running_example(rng, n, 0.6)
+    expr = "R[i,j,k] = A[i,p,q] * B[j,p,r] * C[k,q,r] * D[j,k,r]"
+    ext = {x: n for x in "ijkpqr"}
+    S1, A1 = oc.nary_direct(expr, ops, ext)
+    S2, A2 = oc.nary_einsum(expr, ops, ext)
+    np.testing.assert_allclose(S2, S1, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(A2, A1, rtol=1e-12, atol=1e-13)
+    assert np.all(A2 >= np.abs(S2) - 1e-12) and np.any(A2 > np.abs(S2) + 1e-9)      # signs do cancel somewhere
+
+    dims = (4, 3, 2, 3)
+    X = rand_coo(rng, dims, 0.3)
+    fac = {"B": rng.standard_normal((3, 2)), "C": rng.standard_normal((2, 2)), "D": rng.standard_normal((3, 2))}
+    expr4 = "M[i,r] = X[i,j,k,l] * B[j,r] * C[k,r] * D[l,r]"
+    ext4 = {"i": 4, "j": 3, "k": 2, "l": 3, "r": 2}
+    S1, A1 = oc.nary_direct(expr4, dict(fac, X=X), ext4)
+    S2, A2 = oc.nary_einsum(expr4, dict(fac, X=X), ext4)
+    np.testing.assert_allclose(S2, S1, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(A2, A1, rtol=1e-12, atol=1e-13)
+
+    I3 = rand_coo(rng, (3, 4, 3), 0.5)
+    L = rand_coo(rng, (3, 2), 0.5)
+    L = (L[0], np.ones_like(L[1]))
+    Cm, Pm = rng.standard_normal((4, 2)), rng.standard_normal((3, 4))
+    exprm = "E[k,i,m] = I[k,u,v] * C[u,i] * P[v,m] * L[k,i]"
+    extm = {"k": 3, "u": 4, "v": 3, "i": 2, "m": 4}
+    S1, A1 = oc.nary_direct(exprm, {"I": I3, "C": Cm, "P": Pm, "L": L}, extm)
+    S2, A2 = oc.nary_einsum(exprm, {"I": I3, "C": Cm, "P": Pm, "L": L}, extm)
+    np.testing.assert_allclose(S2, S1, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(A2, A1, rtol=1e-12, atol=1e-13)
+    mask = densify(*L, (3, 2))
+    assert np.all(S2[mask == 0] == 0)                                   # nothing outside the map
+
+    ones = {"X": (X[0], np.ones_like(X[1])), "B": np.ones((3, 2)), "C": np.ones((2, 2)), "D": np.ones((3, 2))}
+    S, A = oc.nary_einsum(expr4, ones, ext4)
+    per_slice = np.bincount(X[0][0], minlength=4)
+    np.testing.assert_array_equal(S, np.repeat(per_slice[:, None], 2, axis=1))
+    np.testing.assert_array_equal(A, S)

@@ -31,9 +31,10 @@ def test_paper_running_example_is_legal_and_reduces_to_2d():
     g, ext = _running_example()
     red = cb.const_schedule_check(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext)
     assert red == [g["reduced_orders"]["X"], g["reduced_orders"]["Y"], 0]
-    # a legal schedule without a kernel family is "unsupported", not "illegal"
-    assert _status(cb.const_plan_create, g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext,
-                   cb.F64) == 2
+    # no hand-written kernel family matches four sparse tensors: the plan binds to the generic executor
+    p = cb.const_plan_create(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext, cb.F64)
+    assert cb.const_plan_family(p) == "tree"
+    assert [cb.const_plan_reduced_order(p, c) for c in range(3)] == [2, 2, 0]
 
 
 def test_paper_running_example_violations():
@@ -106,18 +107,29 @@ def test_other_families_and_modes():
     assert cb.const_plan_family(p) == "ttmc3"
 
 
-def test_unsupported_but_legal():
+def _family(**kw):
+    """Family a descriptor binds to, or the status code when plan creation fails."""
+    try:
+        return cb.const_plan_family(cb.const_plan_create(kw["expression"], kw["tree"], kw["mode_orders"],
+                                                         kw["loop_orders"], kw["extents"], kw["dtype"]))
+    except cb.ConstError as e:
+        return e.status
+
+
+def test_legal_schedules_outside_the_families_run_on_the_generic_executor():
     w = ttmc3_workload((6, 5, 4), 20, 8)
-    mk = lambda **kw: _status(cb.const_plan_create, kw.get("expression", w.expression), kw.get("tree", w.tree),
-                              kw.get("mode_orders", w.mode_orders), kw.get("loop_orders", w.loop_orders),
-                              kw.get("extents", w.extents), kw.get("dtype", cb.F32))
-    assert mk() == 0
-    assert mk(loop_orders=["ijkb", "iajb"]) == 2              # legal, but t would be order 2
-    assert mk(dtype=cb.F64) == 2                              # chain kernels compute in fp32
+    base = dict(expression=w.expression, tree=w.tree, mode_orders=w.mode_orders, loop_orders=w.loop_orders,
+                extents=w.extents, dtype=cb.F32)
+    mk = lambda **kw: _family(**dict(base, **kw))
+    assert mk() == "ttmc3"
+    assert mk(loop_orders=["ijkb", "iajb"]) == "tree"         # legal, but t stays order 2: no hand-written kernel
+    assert mk(dtype=cb.F64) == "tree"                         # the chain kernels compute in fp32
     ext = dict(w.extents); ext["a"] = 12
-    assert mk(extents=ext) == 2                               # rank not 8/16/32
+    assert mk(extents=ext) == "tree"                          # rank not 8/16/32
     assert mk(expression="Y[i,b,a] = X[i,j,k] * U[j,a] * V[k,b]",
-              tree=["T[i,j,b] = X[i,j,k] * V[k,b]", "Y[i,b,a] = T[i,j,b] * U[j,a]"]) == 2   # output layout
+              tree=["T[i,j,b] = X[i,j,k] * V[k,b]", "Y[i,b,a] = T[i,j,b] * U[j,a]"]) == "tree"   # output layout
+    big = dict(w.extents); big["i"] = 1 << 26; big["a"] = 12  # no family (rank 12), and the dense result would hold 2^31 elements or more
+    assert mk(extents=big) == 2                               # beyond every executor: unsupported, not illegal
     assert mk(loop_orders=["ikjb", "ijab"]) == 3              # disagrees with CSF order (i,j,k)
     # contracting j before k is a different tree: legal only with k fused above j, which CSF (i,j,k) forbids
     assert mk(tree=["T[i,k,a] = X[i,j,k] * U[j,a]", "Y[i,a,b] = T[i,k,a] * V[k,b]"],
@@ -126,17 +138,18 @@ def test_unsupported_but_legal():
 
 def test_network_schedule_variants():
     w = network_workload(16, 4, 3)
-    mk = lambda **kw: _status(cb.const_plan_create, w.expression, kw.get("tree", w.tree),
-                              kw.get("mode_orders", w.mode_orders), kw.get("loop_orders", w.loop_orders),
-                              w.extents, kw.get("dtype", cb.F64))
-    assert mk() == 0
-    # scatter-form schedule (U stored i,j,k; W stored k,l,m) is legal but has no kernel here
-    assert mk(mode_orders={"U": (0, 1, 2), "W": (0, 1, 2)}, loop_orders=["ijkl", "iklm"]) == 2
+    mk = lambda **kw: _family(expression=w.expression, tree=kw.get("tree", w.tree),
+                              mode_orders=kw.get("mode_orders", w.mode_orders),
+                              loop_orders=kw.get("loop_orders", w.loop_orders), extents=w.extents,
+                              dtype=kw.get("dtype", cb.F64))
+    assert mk() == "network"
+    # scatter-form schedule (U stored i,j,k; W stored k,l,m): legal, generic executor
+    assert mk(mode_orders={"U": (0, 1, 2), "W": (0, 1, 2)}, loop_orders=["ijkl", "iklm"]) == "tree"
     # not fused over i: T stays order 3
-    assert mk(loop_orders=["ikjl", "lmik"]) == 2               # legal, but T keeps all three modes
+    assert mk(loop_orders=["ikjl", "lmik"]) == "tree"          # legal, T keeps all three modes (a global workspace)
     assert mk(loop_orders=["ikjl", "imlk"]) == 3               # W stored (l,m,k): m may not precede l
-    assert mk(mode_orders={"U": (0, 2, 1), "W": (2, 1, 0)}, loop_orders=["ikjl", "imlk"]) == 2   # W as (m,l,k)
-    assert mk(dtype=cb.F32) == 2
+    assert mk(mode_orders={"U": (0, 2, 1), "W": (2, 1, 0)}, loop_orders=["ikjl", "imlk"]) == "tree"   # W as (m,l,k)
+    assert mk(dtype=cb.F32) == "tree"
 
 
 def test_malformed_descriptors():
