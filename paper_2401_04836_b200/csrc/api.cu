@@ -41,12 +41,12 @@ bool csf_matches(const const_csf *c, const PlanDesc &d, const std::string &name,
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-std::atomic<int> g_spin_limit{0}, g_withhold{0};
+std::atomic<int> g_spin_limit{0}, g_withhold{0}, g_variant{0};
 
 }  // namespace
 
 namespace cb {
-DebugKnobs debug_knobs() { return DebugKnobs{g_spin_limit.load(), g_withhold.load()}; }
+DebugKnobs debug_knobs() { return DebugKnobs{g_spin_limit.load(), g_withhold.load(), g_variant.load()}; }
 }  // namespace cb
 
 extern "C" {
@@ -387,6 +387,7 @@ const_status_t const_debug_set(int what, int64_t value) {
     switch (what) {
         case 0: g_spin_limit.store((int)value); return CONST_OK;
         case 1: g_withhold.store(value != 0); return CONST_OK;
+        case 2: g_variant.store((int)value); return CONST_OK;
     }
     return CONST_ERR_INVALID_ARG;
 }

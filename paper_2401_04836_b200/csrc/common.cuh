@@ -129,6 +129,7 @@ private:
 struct DebugKnobs {
     int spin_limit;      // polls before a wait gives up (0: the kernel's own default)
     int withhold;        // nonzero: producers do not publish / the tensor-core stage does not commit
+    int variant;         // kernel variant to launch where a launcher keeps several for measurement (0: the default)
 };
 DebugKnobs debug_knobs();
 

@@ -19,7 +19,7 @@
 // becomes the limit.  So both phases sweep their fibre range in chunks: the chunk's (coordinate,
 // value) pairs are copied into shared memory with coalesced loads as 16-byte records, and a group
 // of GL lanes then walks one fibre, every lane of the group reading the same record (one broadcast
-// 128-bit shared-memory load) and its own VPT = 8/GL entries of the V row (producer, contiguous
+// 128-bit shared-memory load) and its own LT/GL entries of the V row (producer, contiguous
 // in global memory) or of the T row (consumer, contiguous in shared memory).  The partial sums of
 // the (l, m) fibres are combined with fp64 atomic adds on Z.
 #include "common.cuh"
@@ -27,7 +27,7 @@
 namespace cb {
 namespace {
 
-constexpr int LT = 8;          // l values per block
+constexpr int kMaxLT = 32;     // most l values a block may own
 constexpr int kThreads = 512;
 constexpr int RB = 2048;       // records staged per chunk (a multiple of the block size)
 constexpr int FPMAX = 1024;    // fibre descriptors staged per batch
@@ -108,12 +108,14 @@ __device__ __forceinline__ void sweep(const Csf3d &x, int32_t fA, int32_t fB, co
     }
 }
 
-template <int IS, int GL>
+template <int IS, int LT, int GL>
 __global__ void __launch_bounds__(kThreads)
 network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restrict__ Z, int n_k, int n_l, int n_m,
                int v_vec_ok) {
-    constexpr int VPT = 8 / GL;                    // entries of a V row (producer) or T row (consumer) per lane
-    static_assert(LT == 8 && IS == 8 && (VPT == 1 || VPT == 2 || VPT == 4), "a lane group covers the 8 l of the tile or the 8 i of the strip");
+    constexpr int VPT_P = LT / GL;                 // entries of a V row per lane (producer)
+    constexpr int VPT_C = IS / GL;                 // entries of a T row per lane (consumer)
+    static_assert(LT % GL == 0 && IS % GL == 0 && LT <= kMaxLT && (VPT_P == 1 || VPT_P % 2 == 0) &&
+                  (VPT_C == 1 || VPT_C % 2 == 0), "a lane group covers the l of the tile or the i of the strip");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int TL = n_k * IS + 2;                   // doubles per l plane; the +2 staggers the banks of the 8 planes
     double *T = reinterpret_cast<double *>(smem_raw);                               // [LT][n_k][IS]
@@ -155,20 +157,20 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
 
     // ---- producer: T[l][k][ii] = sum_j U[i,k,j] * V[j, l0 + l]
     {
-        const int lq = q * VPT;                    // first l of this lane, relative to the tile
+        const int lq = q * VPT_P;                    // first l of this lane, relative to the tile
         const double *vcol = V + l0 + lq;
-        const bool vec = v_vec_ok && VPT >= 2 && l0 + lq + VPT <= n_l;     // whole lane inside the row, 16-byte aligned
+        const bool vec = v_vec_ok && VPT_P >= 2 && l0 + lq + VPT_P <= n_l;     // whole lane inside the row, 16-byte aligned
         sweep<GL>(u, s_pos[0], s_pos[IS], st, [&](int32_t f, int32_t k, const Rec *recs, int n) {
             int ii = 0;
             while (ii + 1 < IS && s_pos[ii + 1] <= f) ++ii;
-            double a[VPT], b[VPT];                 // two accumulator sets: consecutive records alternate
+            double a[VPT_P], b[VPT_P];                 // two accumulator sets: consecutive records alternate
 #pragma unroll
-            for (int c = 0; c < VPT; ++c) a[c] = b[c] = 0.0;
+            for (int c = 0; c < VPT_P; ++c) a[c] = b[c] = 0.0;
             if (vec) {
-                auto row_fma = [&](const Rec &r, double (&acc)[VPT]) {
+                auto row_fma = [&](const Rec &r, double (&acc)[VPT_P]) {
                     const double2 *row = reinterpret_cast<const double2 *>(vcol + (size_t)r.c * n_l);
 #pragma unroll
-                    for (int c = 0; c < VPT / 2; ++c) {
+                    for (int c = 0; c < VPT_P / 2; ++c) {
                         const double2 v = __ldg(row + c);
                         acc[2 * c] = fma(r.v, v.x, acc[2 * c]);
                         acc[2 * c + 1] = fma(r.v, v.y, acc[2 * c + 1]);
@@ -186,23 +188,23 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
                     const Rec r0 = recs[e];
                     const double *row = vcol + (size_t)r0.c * n_l;
 #pragma unroll
-                    for (int c = 0; c < VPT; ++c)
+                    for (int c = 0; c < VPT_P; ++c)
                         if (l0 + lq + c < n_l) a[c] = fma(r0.v, __ldg(row + c), a[c]);
                 }
             }
             double *t = T + (size_t)lq * TL + k * IS + ii;
 #pragma unroll
-            for (int c = 0; c < VPT; ++c) t[c * TL] += a[c] + b[c];
+            for (int c = 0; c < VPT_P; ++c) t[c * TL] += a[c] + b[c];
         });
     }
     // (the sweep ends with a block barrier: T is complete)
 
     // ---- consumer: Z[i,m] += sum_{k in fibre (l,m)} T[l][k][ii] * W[l,m,k]
     {
-        const int iq = q * VPT;                    // first slice of this lane, relative to the strip
-        int32_t rows[VPT];
+        const int iq = q * VPT_C;                    // first slice of this lane, relative to the strip
+        int32_t rows[VPT_C];
 #pragma unroll
-        for (int c = 0; c < VPT; ++c) {
+        for (int c = 0; c < VPT_C; ++c) {
             const int s = strip * IS + iq + c;
             rows[c] = s < u.n0 ? __ldg(u.crd0 + s) : -1;
         }
@@ -210,14 +212,14 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
             int node = 0;
             while (node + 1 < nodes && w_pos[node + 1] <= f) ++node;
             const double *t = T + (size_t)w_l[node] * TL + iq;
-            double a[VPT], b[VPT];
+            double a[VPT_C], b[VPT_C];
 #pragma unroll
-            for (int c = 0; c < VPT; ++c) a[c] = b[c] = 0.0;
-            auto row_fma = [&](const Rec &r, double (&acc)[VPT]) {
+            for (int c = 0; c < VPT_C; ++c) a[c] = b[c] = 0.0;
+            auto row_fma = [&](const Rec &r, double (&acc)[VPT_C]) {
                 const double *row = t + r.c * IS;
-                if constexpr (VPT >= 2) {
+                if constexpr (VPT_C >= 2) {
 #pragma unroll
-                    for (int c = 0; c < VPT / 2; ++c) {
+                    for (int c = 0; c < VPT_C / 2; ++c) {
                         const double2 tv = *reinterpret_cast<const double2 *>(row + 2 * c);
                         acc[2 * c] = fma(tv.x, r.v, acc[2 * c]);
                         acc[2 * c + 1] = fma(tv.y, r.v, acc[2 * c + 1]);
@@ -234,7 +236,7 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
             }
             if (e < n) row_fma(recs[e], a);
 #pragma unroll
-            for (int c = 0; c < VPT; ++c)
+            for (int c = 0; c < VPT_C; ++c)
                 if (rows[c] >= 0) atomicAdd(Z + (size_t)rows[c] * n_m + m, a[c] + b[c]);
         });
     }
@@ -242,16 +244,15 @@ network_kernel(Csf3d u, const double *__restrict__ V, Csf3d w, double *__restric
 
 }  // namespace
 
-const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z, int64_t n_i,
-                           int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m, int32_t *, cudaStream_t stream) {
-    (void)n_j;
-    constexpr int IS = 8, GL = 4;   // lanes per fibre: 2 -> 5.8 ms, 4 -> 4.8 ms, 8 -> 6.2 ms on the benchmark network
-    CB_CUDA(cudaMemsetAsync(Z, 0, sizeof(double) * n_i * n_m, stream));
-    if (U->nnz == 0 || W->nnz == 0) return CONST_OK;
+namespace {
+
+template <int IS, int LT, int GL>
+const_status_t launch_network(const const_csf *U, const double *V, const const_csf *W, double *Z, int64_t n_k,
+                              int64_t n_l, int64_t n_m, cudaStream_t stream) {
     const size_t t_doubles = ((size_t)LT * (n_k * IS + 2) + 1) / 2 * 2;
     const size_t smem = sizeof(double) * t_doubles + sizeof(Rec) * RB + sizeof(int32_t) * (2 * FPMAX + 1);
     if (smem > 220 * 1024 || n_l > (1ll << 30) || n_m > (1ll << 30)) return CONST_ERR_WORKSPACE;
-    auto kernel = network_kernel<IS, GL>;
+    auto kernel = network_kernel<IS, LT, GL>;
     // the requested size depends on n_k: raise the limit once per device to the most a block may have
     static PerDeviceOnce attr_once;
     CB_CUDA(once_per_device(attr_once, [&] { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024); }));
@@ -263,6 +264,24 @@ const_status_t run_network(const const_csf *U, const double *V, const const_csf 
               kernel<<<grid, kThreads, smem, stream>>>(u, V, w, Z, (int)n_k, (int)n_l, (int)n_m, v_vec_ok));
     CB_CUDA(cudaGetLastError());
     return CONST_OK;
+}
+
+}  // namespace
+
+const_status_t run_network(const const_csf *U, const double *V, const const_csf *W, double *Z, int64_t n_i,
+                           int64_t n_j, int64_t n_k, int64_t n_l, int64_t n_m, int32_t *, cudaStream_t stream) {
+    (void)n_j;
+    CB_CUDA(cudaMemsetAsync(Z, 0, sizeof(double) * n_i * n_m, stream));
+    if (U->nnz == 0 || W->nnz == 0) return CONST_OK;
+    // tile shape (slices per strip, l per tile, lanes per fibre); the variants are kept for measurement
+    switch (debug_knobs().variant) {
+        case 1: return launch_network<8, 16, 4>(U, V, W, Z, n_k, n_l, n_m, stream);
+        case 2: return launch_network<16, 8, 4>(U, V, W, Z, n_k, n_l, n_m, stream);
+        case 3: return launch_network<8, 16, 8>(U, V, W, Z, n_k, n_l, n_m, stream);
+        case 4: return launch_network<16, 8, 8>(U, V, W, Z, n_k, n_l, n_m, stream);
+        case 5: return launch_network<4, 16, 4>(U, V, W, Z, n_k, n_l, n_m, stream);
+        default: return launch_network<8, 8, 4>(U, V, W, Z, n_k, n_l, n_m, stream);
+    }
 }
 
 }  // namespace cb
