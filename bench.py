@@ -214,7 +214,7 @@ def measure_machine_peaks(cb, local_rank):
     sampler.start()
     out = {}
     for name, kind in (("fp32_fma_tflops", cb.BENCH_FP32_FMA), ("fp64_fma_tflops", cb.BENCH_FP64_FMA),
-                       ("tf32_mma_tflops", cb.BENCH_TF32_MMA)):
+                       ("fp64_mma_tflops", cb.BENCH_FP64_MMA), ("tf32_mma_tflops", cb.BENCH_TF32_MMA)):
         best = 0.0
         for _ in range(3):
             ms, work = cb.const_microbench(kind, repeats=20 if kind != cb.BENCH_TF32_MMA else 5)
@@ -223,7 +223,7 @@ def measure_machine_peaks(cb, local_rank):
     clocks = sampler.stop()
     out["sm_mhz_during"] = clocks["sm_mhz"]
     out["how"] = ("const_microbench: 8 independent FMA chains per thread on 8 x 256 threads per SM; tcgen05.mma "
-                  "kind::tf32 M128 N256 K8 from shared memory, one block per SM; best of 3")
+                  "kind::tf32 M128 N256 K8 from shared memory, one block per SM; mma.sync m8n8k4 f64 from registers; best of 3")
     return out
 
 

@@ -284,8 +284,10 @@ const char *const_status_string(const_status_t status);
  * tensor-core stage).  what = 0: number of polls after which a wait gives up (0 restores the defaults);
  * what = 1: value != 0 withholds the signal those waits wait for -- sort tiles do not publish their
  * counts, the tensor-core stage issues and commits nothing -- so that every such wait runs out, the
- * kernel records CONST_ERR_TIMEOUT, skips its stores and returns normally.  Process-wide; not for
- * production use.  CONST_ERR_INVALID_ARG for an unknown `what` or a value outside [0, 2^31).
+ * kernel records CONST_ERR_TIMEOUT, skips its stores and returns normally;
+ * what = 2: which of the tile shapes a launcher keeps for measurement is launched (0: the default; the
+ * two-contraction network has variants 1..5, every one of them computes the same result).  Process-wide; not
+ * for production use.  CONST_ERR_INVALID_ARG for an unknown `what` or a value outside [0, 2^31).
  */
 const_status_t const_debug_set(int what, int64_t value);
 
@@ -312,15 +314,16 @@ const_status_t const_profile_read(char *names, int64_t names_bytes, int64_t *lau
  *   CONST_BENCH_FP32_FMA / CONST_BENCH_FP64_FMA   register-only fused multiply-adds on every SM; work in flop;
  *   CONST_BENCH_TF32_MMA     tcgen05.mma kind::tf32, M 128 x N 256 x K 8, operands in shared memory, accumulator
  *                            in tensor memory, one block per SM; work in flop;
+ *   CONST_BENCH_FP64_MMA     mma.sync m8n8k4 in fp64 from registers on every SM (the fp64 matrix path); work in flop;
  *   CONST_BENCH_ROW_GATHER   rows_dev[n] (device, int32 row numbers, e.g. a leaf-level crd array) are gathered
  *                            from a table of table_rows x rank floats (rank 8, 16 or 32) with 128-bit loads, rank / 4
  *                            lanes per row, four rows in flight per lane; work in bytes of rows read.
- * rows_dev, n, table_rows and rank are ignored by the first three kinds.  The call allocates its table and a
+ * rows_dev, n, table_rows and rank are ignored by every kind but the row gather.  The call allocates its table and a
  * status word stream-ordered and frees them before it returns.  CONST_ERR_TIMEOUT if the bounded wait for the
  * tensor pipe gave up.
  */
 typedef enum { CONST_BENCH_FP32_FMA = 0, CONST_BENCH_FP64_FMA = 1, CONST_BENCH_TF32_MMA = 2,
-               CONST_BENCH_ROW_GATHER = 3 } const_microbench_kind_t;
+               CONST_BENCH_ROW_GATHER = 3, CONST_BENCH_FP64_MMA = 4 } const_microbench_kind_t;
 const_status_t const_microbench(int kind, const int32_t *rows_dev, int64_t n, int64_t table_rows, int rank, int repeats,
                                 void *stream, double *ms_per_launch, double *work_per_launch);
 

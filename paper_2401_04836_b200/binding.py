@@ -262,7 +262,7 @@ def const_csf_work_lists(csf: CsfHandle):
             _dev_to_torch(it.value, 4 * n_items.value, torch.int32).reshape(-1, 4))
 
 
-BENCH_FP32_FMA, BENCH_FP64_FMA, BENCH_TF32_MMA, BENCH_ROW_GATHER = 0, 1, 2, 3
+BENCH_FP32_FMA, BENCH_FP64_FMA, BENCH_TF32_MMA, BENCH_ROW_GATHER, BENCH_FP64_MMA = 0, 1, 2, 3, 4
 
 
 def const_microbench(kind: int, rows=None, table_rows: int = 0, rank: int = 0, repeats: int = 5, stream=None):

@@ -32,6 +32,24 @@ __global__ void __launch_bounds__(kFmaThreads) fma_peak_kernel(T a, T b, T *sink
     if (s == (T)123456789) sink[0] = s;                                   // keeps the chains alive; practically never true
 }
 
+// ---- fp64 tensor path: mma.sync m8n8k4 (the only fp64 matrix instruction; tcgen05 has no fp64 kind) ----
+constexpr int kDmmaIters = 4096, kDmmaChains = 4;
+__global__ void __launch_bounds__(kFmaThreads) dmma_peak_kernel(double a, double b, double *sink) {
+    double c[kDmmaChains][2];
+#pragma unroll
+    for (int k = 0; k < kDmmaChains; ++k) c[k][0] = c[k][1] = a * (double)(threadIdx.x + k);
+    for (int it = 0; it < kDmmaIters; ++it) {
+#pragma unroll
+        for (int k = 0; k < kDmmaChains; ++k)
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                         : "+d"(c[k][0]), "+d"(c[k][1]) : "d"(a), "d"(b));
+    }
+    double s = 0;
+#pragma unroll
+    for (int k = 0; k < kDmmaChains; ++k) s += c[k][0] + c[k][1];
+    if (s == 123456789.0) sink[0] = s;
+}
+
 // ---- tf32 tensor pipe: M = 128, N = 256, K = 8 per instruction, the largest single-CTA shape ----
 constexpr int kMmaM = 128, kMmaN = 256;
 constexpr int kMmaPerBlock = 4096;
@@ -116,7 +134,7 @@ using namespace cb;
 extern "C" const_status_t const_microbench(int kind, const int32_t *rows_dev, int64_t n, int64_t table_rows, int rank,
                                            int repeats, void *stream_v, double *ms_per_launch, double *work_per_launch) {
     if (!ms_per_launch || !work_per_launch || repeats < 1 || repeats > 1000 || kind < CONST_BENCH_FP32_FMA ||
-        kind > CONST_BENCH_ROW_GATHER)
+        kind > CONST_BENCH_FP64_MMA)
         return CONST_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     int dev = 0, sms = 0;
@@ -144,11 +162,15 @@ extern "C" const_status_t const_microbench(int kind, const int32_t *rows_dev, in
                 fma_peak_kernel<double><<<sms * 8, kFmaThreads, 0, stream>>>(1.0000001, 1e-9, reinterpret_cast<double *>(scratch));
                 work = 2.0 * kFmaChains * kFmaIters * kFmaThreads * (double)(sms * 8);
                 break;
+            case CONST_BENCH_FP64_MMA:
+                dmma_peak_kernel<<<sms * 8, kFmaThreads, 0, stream>>>(1.0000001, 1e-9, reinterpret_cast<double *>(scratch));
+                work = 2.0 * 8 * 8 * 4 * kDmmaChains * (double)kDmmaIters * (kFmaThreads / 32) * (double)(sms * 8);
+                break;
             case CONST_BENCH_TF32_MMA:
                 mma_peak_kernel<<<sms, 128, kMmaABytes + kMmaBBytes, stream>>>(reinterpret_cast<int32_t *>(scratch), umma::kMbarPolls);
                 work = 2.0 * kMmaM * kMmaN * 8 * (double)kMmaPerBlock * sms;
                 break;
-            default: {
+            case CONST_BENCH_ROW_GATHER: {
                 const float *table = scratch + 64;
                 if (rank == 8) gather_peak_kernel<8, 4><<<sms * 8, 256, 0, stream>>>(rows_dev, table, n, table_rows, scratch);
                 else if (rank == 16) gather_peak_kernel<16, 4><<<sms * 8, 256, 0, stream>>>(rows_dev, table, n, table_rows, scratch);
