@@ -173,13 +173,15 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
+    interval_ms = 20
+
     def __init__(self, gpu_index):
         self.rows, self.proc, self.gpu = [], None, gpu_index
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                          "--format=csv,noheader,nounits", "-lms", str(self.interval_ms)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
@@ -187,15 +189,19 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append([time.monotonic()] + [x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Ends the sampling; the summary covers the samples taken between the monotonic times t0 and t1
+        (all of them when no window is given, or when the window holds none)."""
         if self.proc:
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=2)
             except Exception:
                 self.proc.kill()
+        window = [r[1:] for r in self.rows if t0 is not None and t0 <= r[0] <= t1]
+        self.rows = window if window else [r[1:] for r in self.rows]
         sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
         mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -273,6 +279,10 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the clock record starts before the warm-up, so that the start-up of nvidia-smi (which takes driver locks) is
+    # over when the timed region begins; only the samples taken inside the timed region are summarised
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     # warm-up (also sizes the stream-ordered memory pool)
     level_sizes, bins, gather = None, None, None
     for _ in range(args.warmup):
@@ -338,13 +348,16 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
         return total, per_step, per_exec
 
     # ---- timed region: device-resident inputs ----
-    sampler = ClockSampler(torch.cuda.current_device())
-    sampler.start()
+    import gc
     cb.const_profile_enable(True)
+    gc.disable()
+    t_begin = time.monotonic()
     total_ms, per_step, per_exec = timed_loop()
+    t_end = time.monotonic()
+    gc.enable()
     prof = cb.const_profile_read()
     cb.const_profile_enable(False)
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
     exec_ms = float(np.mean(per_exec))
     ms_per_step = total_ms / steps
     ms_per_step, total_flops = aggregate_over_ranks(ms_per_step, flops, dist, "cuda")
@@ -487,9 +500,11 @@ def main():
     ap.add_argument("--tensor-stage", type=int, default=-1,
                     help="TTMc: 1 = dense per-slice stage on the tensor cores, 0 = on the FMA pipes, -1 = library default")
     ap.add_argument("--bins", default="", help="light_max,heavy_max,chunk nonzero thresholds of the load balancer (default: the library's)")
+    ap.add_argument("--smi-ms", type=int, default=20, help="sampling interval of the clock record (nvidia-smi -lms)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernels)")
     args = ap.parse_args()
+    ClockSampler.interval_ms = max(5, args.smi_ms)
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))

@@ -115,6 +115,18 @@ const_status_t const_csf_build_noalloc(int order, const int64_t *dims, int64_t n
                                        int32_t *const *pos_out_dev, int32_t *const *crd_out_dev, void *vals_out_dev,
                                        int64_t *level_sizes);
 
+/*
+ * Dense array -> CSF (Sec. 2.1: the nonzeros of a result are the entries that are not zero).  dense_dev is a
+ * row-major device array with extents dims[0..order) of `dtype`; every entry that compares unequal to zero
+ * becomes a stored nonzero (so -0.0 is dropped and NaN is kept), the rest as for const_csf_build.  This is how
+ * the dense result of one network becomes a sparse operand of the next, e.g. the 3-index integrals E of
+ * Sec. 5.1 Eq. 1 as the two CSF operands of the 4-index contraction of Eq. 3, and how a result is handed out
+ * in CSF form.  The call waits for the stream twice (the number of nonzeros, then the level sizes).
+ * CONST_ERR_UNSUPPORTED for more than 2^40 cells or 2^31 - 2 nonzeros.
+ */
+const_status_t const_csf_from_dense(int order, const int64_t *dims, const void *dense_dev, const_dtype_t dtype,
+                                    const int *mode_order, void *stream, const_csf_t **out);
+
 /* Borrowed device pointers of one level (valid until const_destroy).  *pos has n_{level-1}+1 entries
  * (2 for level 0), *crd has *n entries.  Any output pointer may be NULL. */
 const_status_t const_csf_level(const const_csf_t *csf, int level, const int32_t **pos, const int32_t **crd,

@@ -54,6 +54,8 @@ def load_library():
     vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
     pp = ctypes.POINTER
     lib.const_csf_build.argtypes = [i32, pp(i64), i64, pp(vp), vp, i32, pp(i32), vp, pp(vp)]
+    lib.const_csf_from_dense.argtypes = [i32, pp(i64), vp, i32, pp(i32), vp, pp(vp)]
+    lib.const_csf_from_dense.restype = i32
     lib.const_csf_build_noalloc.argtypes = [i32, pp(i64), i64, pp(vp), vp, i32, pp(i32), vp, pp(vp), pp(vp), vp,
                                             pp(i64)]
     lib.const_csf_build_noalloc.restype = i32
@@ -161,6 +163,22 @@ def const_csf_build(coords, vals, dims: Sequence[int], mode_order: Sequence[int]
     st = lib.const_csf_build(order, dims_a, nnz, cptr, ctypes.c_void_p(vals.data_ptr()), dtype, mo_a,
                              _stream_ptr(stream), ctypes.byref(out))
     _check(st, "const_csf_build")
+    return CsfHandle(out.value, order, dtype)
+
+
+def const_csf_from_dense(dense, mode_order: Sequence[int], stream=None) -> CsfHandle:
+    """dense: contiguous float32/float64 CUDA tensor; its entries that are not zero become the CSF tensor's nonzeros."""
+    import torch
+    lib = load_library()
+    if not dense.is_cuda or not dense.is_contiguous() or dense.dtype not in (torch.float32, torch.float64):
+        raise ValueError("dense must be a contiguous float32/float64 CUDA tensor")
+    order = dense.dim()
+    dtype = F32 if dense.dtype == torch.float32 else F64
+    dims_a = (ctypes.c_int64 * order)(*[int(d) for d in dense.shape])
+    mo_a = (ctypes.c_int * order)(*[int(m) for m in mode_order])
+    out = ctypes.c_void_p()
+    _check(lib.const_csf_from_dense(order, dims_a, ctypes.c_void_p(dense.data_ptr()), dtype, mo_a, _stream_ptr(stream),
+                                    ctypes.byref(out)), "const_csf_from_dense")
     return CsfHandle(out.value, order, dtype)
 
 

@@ -74,6 +74,23 @@ const_status_t const_csf_build(int order, const int64_t *dims, int64_t nnz, cons
     return rc;
 }
 
+const_status_t const_csf_from_dense(int order, const int64_t *dims, const void *dense_dev, const_dtype_t dtype,
+                                    const int *mode_order, void *stream, const_csf_t **out) {
+    if (!out) return CONST_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (order < 2 || order > kMaxOrder || !dims || !dense_dev || !mode_order || (dtype != CONST_F32 && dtype != CONST_F64))
+        return CONST_ERR_INVALID_ARG;
+    bool seen[kMaxOrder] = {false, false, false, false};
+    for (int l = 0; l < order; ++l) {
+        if (mode_order[l] < 0 || mode_order[l] >= order || seen[mode_order[l]] || dims[l] < 1) return CONST_ERR_INVALID_ARG;
+        seen[mode_order[l]] = true;
+    }
+    const_csf *csf = nullptr;
+    const_status_t rc = csf_from_dense_impl(order, dims, dense_dev, dtype, mode_order, static_cast<cudaStream_t>(stream), &csf);
+    if (rc == CONST_OK) *out = csf;
+    return rc;
+}
+
 const_status_t const_csf_build_noalloc(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
                                        const void *vals_dev, const_dtype_t dtype, const int *mode_order, void *stream,
                                        int32_t *const *pos_out_dev, int32_t *const *crd_out_dev, void *vals_out_dev,

@@ -137,6 +137,8 @@ DebugKnobs debug_knobs();
 const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const int32_t *const *coords_dev,
                               const void *vals_dev, const_dtype_t dtype, const int *mode_order,
                               cudaStream_t stream, const_csf **out);
+const_status_t csf_from_dense_impl(int order, const int64_t *dims, const void *dense, const_dtype_t dtype,
+                                   const int *mode_order, cudaStream_t stream, const_csf **out);
 const_status_t csf_rebin(const_csf *csf, cudaStream_t stream);
 const_status_t csf_bin_totals(const_csf *csf);      // fills the host copies n_light .. n_items (waits for the device once)
 void csf_free(const_csf *csf);

@@ -1168,4 +1168,94 @@ const_status_t csf_build_noalloc_impl(int order, const int64_t *dims, int64_t nn
     return CONST_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// const_csf_from_dense: a dense result as a CSF tensor (the entries that are not zero become its
+// nonzeros; Sec. 2.1 defines nz(R) that way), so that the result of one network can be a sparse
+// operand of the next, e.g. E of Sec. 5.1 Eq. 1 feeding the 4-index contraction of Eq. 3.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+struct DenseShape { int64_t dim[kMaxOrder]; int order; };
+
+template <typename T>
+__global__ void __launch_bounds__(256) dense_count(const T *__restrict__ a, int64_t n, unsigned long long *total) {
+    unsigned long long mine = 0;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += stride) mine += a[e] != T(0);
+    mine = __reduce_add_sync(0xffffffffu, (unsigned)mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(total, mine);
+}
+
+// every stored entry gets the next free slot (one atomic per warp and step); the order is arbitrary, the sort
+// of the CSF build establishes the final one
+template <typename T>
+__global__ void __launch_bounds__(256) dense_fill(const T *__restrict__ a, int64_t n, DenseShape sh, int32_t *c0,
+                                                  int32_t *c1, int32_t *c2, int32_t *c3, T *__restrict__ vals,
+                                                  unsigned long long *cursor, unsigned long long capacity) {
+    const int lane = threadIdx.x & 31;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t rounds = (n + stride - 1) / stride;
+    for (int64_t r = 0; r < rounds; ++r) {
+        const int64_t e = r * stride + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        const bool keep = e < n && a[e] != T(0);
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (!m) continue;
+        unsigned long long base = 0;
+        if (lane == __ffs(m) - 1) base = atomicAdd(cursor, (unsigned long long)__popc(m));
+        base = __shfl_sync(0xffffffffu, base, __ffs(m) - 1);
+        if (!keep) continue;
+        const unsigned long long at = base + __popc(m & ((1u << lane) - 1u));
+        if (at >= capacity) continue;                     // cannot happen: the count pass saw the same array
+        int64_t rest = e;
+        int32_t c[kMaxOrder] = {0, 0, 0, 0};
+        for (int d = sh.order - 1; d >= 0; --d) { c[d] = (int32_t)(rest % sh.dim[d]); rest /= sh.dim[d]; }
+        c0[at] = c[0];
+        c1[at] = c[1];
+        if (sh.order > 2) c2[at] = c[2];
+        if (sh.order > 3) c3[at] = c[3];
+        vals[at] = a[e];
+    }
+}
+
+}  // namespace
+
+const_status_t csf_from_dense_impl(int order, const int64_t *dims, const void *dense, const_dtype_t dtype,
+                                   const int *mode_order, cudaStream_t stream, const_csf **out) {
+    int64_t n = 1;
+    DenseShape sh;
+    sh.order = order;
+    for (int d = 0; d < kMaxOrder; ++d) sh.dim[d] = 1;
+    for (int d = 0; d < order; ++d) {
+        sh.dim[d] = dims[d];
+        if (n > (1ll << 40) / dims[d]) return CONST_ERR_UNSUPPORTED;
+        n *= dims[d];
+    }
+    Scratch tmp(stream);
+    unsigned long long *counters = nullptr;
+    CB_CUDA(tmp.alloc((void **)&counters, 64));
+    CB_CUDA(cudaMemsetAsync(counters, 0, 64, stream));
+    const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    if (dtype == CONST_F32) dense_count<float><<<blocks, 256, 0, stream>>>((const float *)dense, n, counters);
+    else dense_count<double><<<blocks, 256, 0, stream>>>((const double *)dense, n, counters);
+    unsigned long long h_nnz = 0;
+    CB_CUDA(cudaMemcpyAsync(&h_nnz, counters, sizeof(h_nnz), cudaMemcpyDeviceToHost, stream));
+    CB_CUDA(wait_stream(stream));
+    if (h_nnz >= 2147483647ull) return CONST_ERR_UNSUPPORTED;
+    const int64_t nnz = (int64_t)h_nnz;
+    int32_t *c[kMaxOrder] = {nullptr, nullptr, nullptr, nullptr};
+    void *vals = nullptr;
+    for (int d = 0; d < order; ++d) CB_CUDA(tmp.alloc((void **)&c[d], sizeof(int32_t) * std::max<int64_t>(nnz, 1)));
+    CB_CUDA(tmp.alloc(&vals, (dtype == CONST_F32 ? 4 : 8) * std::max<int64_t>(nnz, 1)));
+    if (nnz > 0) {
+        if (dtype == CONST_F32)
+            dense_fill<float><<<blocks, 256, 0, stream>>>((const float *)dense, n, sh, c[0], c[1], c[2], c[3], (float *)vals,
+                                                          counters + 1, h_nnz);
+        else
+            dense_fill<double><<<blocks, 256, 0, stream>>>((const double *)dense, n, sh, c[0], c[1], c[2], c[3],
+                                                           (double *)vals, counters + 1, h_nnz);
+        CB_CUDA(cudaGetLastError());
+    }
+    return csf_build_impl(order, dims, nnz, c, vals, dtype, mode_order, stream, out);
+}
+
 }  // namespace cb
