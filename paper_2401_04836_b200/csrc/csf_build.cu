@@ -96,6 +96,9 @@ constexpr int kRsItems = 16;
 constexpr int kRsTile = kRsThreads * kRsItems;     // 4096 keys per tile
 constexpr int kRsWarps = kRsThreads / 32;
 constexpr int kSpinLimit = 1 << 21;
+// Distance, in tiles, of the pass kernel's L2 prefetch: half a wave of its resident blocks (148 SMs x 3).  Measured on
+// 38.5 M nonzeros: none 0.326 ms per pass, 56 to 444 tiles 0.311 ms, 888 and more 0.336 ms (evicted before use).
+constexpr int kRsAheadTiles = 222;
 // A tile's state for one digit is one 64-bit word: the count in the low half; in the high half
 // (pass number << 2) | flag, flag 1 = the tile's own count, flag 2 = the count summed over this and
 // every earlier tile.  A word counts only if it carries the current pass number, so the array is
@@ -126,7 +129,7 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
                                                             const V *__restrict__ vin, V *__restrict__ vout, int64_t n,
                                                             int shift, const uint32_t *__restrict__ digit_base,
                                                             unsigned long long *status, uint32_t *counter,
-                                                            int32_t *err, unsigned epoch, int spin_limit, int withhold) {
+                                                            int32_t *err, unsigned epoch, int spin_limit, int withhold, int ahead_tiles) {
     constexpr int kBins = 1 << BITS;
     constexpr unsigned kDigitMask = kBins - 1;
     constexpr int DPT = kBins / kRsThreads;
@@ -152,6 +155,19 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     if (tile_base >= n) return;                       // never happens: the grid has exactly ceil(n / tile) blocks
     const int64_t left = n - tile_base;
     const int nvalid = left < kRsTile ? (int)left : kRsTile;
+
+    // A tile that will be taken soon (half a wave of resident blocks ahead) is requested into L2 now, so that the
+    // loads of the block that takes it find it there instead of in DRAM.
+    {
+        const int64_t ahead = tile_base + (int64_t)ahead_tiles * kRsTile;
+        const int64_t kb = ahead * (int64_t)sizeof(uint64_t) + (int64_t)threadIdx.x * 128;       // keys: 32 KB = 256 lines
+        if (ahead + kRsTile <= n) {
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(reinterpret_cast<const char *>(kin) + kb));
+            const int64_t vb = ahead * (int64_t)sizeof(V) + (int64_t)threadIdx.x * 128;
+            if ((int64_t)threadIdx.x * 128 < (int64_t)kRsTile * (int64_t)sizeof(V))
+                asm volatile("prefetch.global.L2 [%0];" :: "l"(reinterpret_cast<const char *>(vin) + vb));
+        }
+    }
 
     // this thread's slots of the tile: local indices mine + 32 i
     const int mine = warp * (32 * kRsItems) + lane;
@@ -749,7 +765,8 @@ const_status_t launch_onesweep(const uint64_t *kin, uint64_t *kout, const V *vin
     CB_LAUNCH("rs_onesweep", stream,
               rs_onesweep<V, BITS><<<(unsigned)ntiles, kRsThreads, dyn, stream>>>(
                   kin, kout, vin, vout, n, shift, digit_base, b.tile_status, counter, status, epoch,
-                  knobs.spin_limit > 0 ? knobs.spin_limit : kSpinLimit, knobs.withhold));
+                  knobs.spin_limit > 0 ? knobs.spin_limit : kSpinLimit, knobs.withhold,
+                  kRsAheadTiles));
     return CONST_OK;
 }
 
