@@ -33,6 +33,8 @@ namespace {
 
 __device__ __forceinline__ float4 ldg4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 
+constexpr int kStreamAhead = 256;   // nonzeros between the L2 prefetch of a line of the leaf arrays and its use
+
 __device__ __forceinline__ void fma4(float4 &t, float x, const float4 &v) {
     t.x = fmaf(x, v.x, t.x);
     t.y = fmaf(x, v.y, t.y);
@@ -154,6 +156,10 @@ __device__ __forceinline__ void phase1(const Csf3 &x, const float *__restrict__ 
                 xn = __ldg(reinterpret_cast<const float4 *>(x.vals + m0 + 4));
             }
             for (int32_t p = m0; p < m1; p += 4) {
+                if (q == 0 && ((p >> 2) & 7) == 0 && p + kStreamAhead < m1) {      // once per 128-byte line of the leaf arrays
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(x.crd2 + p + kStreamAhead));
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(x.vals + p + kStreamAhead));
+                }
                 float4 w0 = v0, w1 = v1, w2 = v2, w3 = v3, xw = xn;
                 if (p + 4 < m1) {                                 // gathers of the next block
                     w0 = ldg4(F2q + (size_t)kn.x * R3); w1 = ldg4(F2q + (size_t)kn.y * R3);

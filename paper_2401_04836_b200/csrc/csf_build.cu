@@ -366,6 +366,14 @@ constexpr int kCpThreads = 256;
 constexpr int kCpIters = 8;                                   // 32-element steps per warp
 constexpr int kCpTile = kCpThreads * kCpIters;                // 2048 elements per block
 constexpr int kCpLevels = kMaxOrder - 1;                      // levels that need a scan (all but the leaf level)
+constexpr int kCpAheadTiles = 592;                            // L2 prefetch distance of the one-shot tile kernels (half a wave)
+
+// Requests the keys of the tile `kCpAheadTiles` after this block's into L2 (threads 0..127 take one line each).
+__device__ __forceinline__ void prefetch_tile_ahead(const uint64_t *__restrict__ keys, int64_t n) {
+    const int64_t first = ((int64_t)blockIdx.x + kCpAheadTiles) * kCpTile;
+    if (threadIdx.x < kCpTile * (int)sizeof(uint64_t) / 128 && first + kCpTile <= n)
+        asm volatile("prefetch.global.L2 [%0];" :: "l"(reinterpret_cast<const char *>(keys + first) + threadIdx.x * 128));
+}
 
 struct LevelShifts { int shift[kMaxOrder]; int order; };
 
@@ -408,6 +416,7 @@ __global__ void __launch_bounds__(kCpThreads) csf_count(const uint64_t *__restri
                                                        uint32_t *__restrict__ block_counts, int32_t *status) {
     __shared__ uint32_t sh[kCpLevels];
     if (threadIdx.x < kCpLevels) sh[threadIdx.x] = 0;
+    prefetch_tile_ahead(keys, n);
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t cnt[kCpLevels] = {0, 0, 0};
@@ -479,6 +488,7 @@ __global__ void __launch_bounds__(kCpThreads) csf_scatter(const uint64_t *__rest
                                                          const uint32_t *__restrict__ block_base, CsfArrays out) {
     __shared__ uint32_t wcnt[kCpThreads / 32][kCpLevels];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    prefetch_tile_ahead(keys, n);
     uint64_t key[kCpIters];
     unsigned bal[kCpIters][kCpLevels];
     uint32_t cnt[kCpLevels] = {0, 0, 0};
