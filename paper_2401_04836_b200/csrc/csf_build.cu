@@ -436,45 +436,88 @@ __global__ void __launch_bounds__(kCpThreads) csf_count(const uint64_t *__restri
     if (threadIdx.x < kCpLevels) block_counts[(int64_t)blockIdx.x * kCpLevels + threadIdx.x] = sh[threadIdx.x];
 }
 
-// In-place exclusive scan of per-block counts (one block); totals[l] receives the level sizes.
-__global__ void __launch_bounds__(1024) csf_scan_blocks(uint32_t *block_counts, int64_t nblocks, uint32_t *totals) {
-    __shared__ uint32_t wsum[32][kCpLevels];
-    __shared__ uint32_t carry[kCpLevels];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x < kCpLevels) carry[threadIdx.x] = 0;
+// In-place exclusive scan of the per-block counts, in two launches: every scan block adds up its chunk of
+// kScanChunk counts; then every scan block adds the sums of the chunks before its own (a few dozen numbers) and
+// scans its chunk.  totals[l] receives the level sizes.  `partials` has room for kCpLevels numbers per chunk.
+constexpr int kScanThreads = 256, kScanPer = 4, kScanChunk = kScanThreads * kScanPer;
+
+__device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t *sh) {     // sum over the block, result in every thread
+    v = __reduce_add_sync(0xffffffffu, v);
     __syncthreads();
-    for (int64_t base = 0; base < nblocks; base += 1024) {
-        int64_t b = base + threadIdx.x;
-        uint32_t v[kCpLevels], inc[kCpLevels];
-#pragma unroll
-        for (int l = 0; l < kCpLevels; ++l) {
-            v[l] = b < nblocks ? block_counts[b * kCpLevels + l] : 0;
-            inc[l] = v[l];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                uint32_t t = __shfl_up_sync(0xffffffffu, inc[l], off);
-                if (lane >= off) inc[l] += t;
-            }
-            if (lane == 31) wsum[warp][l] = inc[l];
-        }
-        __syncthreads();
-#pragma unroll
-        for (int l = 0; l < kCpLevels; ++l) {
-            uint32_t wb = 0;
-            for (int w = 0; w < warp; ++w) wb += wsum[w][l];
-            if (b < nblocks) block_counts[b * kCpLevels + l] = carry[l] + wb + inc[l] - v[l];
-        }
-        __syncthreads();
-        if (threadIdx.x == 1023)
-            for (int l = 0; l < kCpLevels; ++l) {
-                uint32_t wb = 0;
-                for (int w = 0; w < 31; ++w) wb += wsum[w][l];
-                carry[l] += wb + inc[l];
-            }
-        __syncthreads();
-    }
-    if (threadIdx.x < kCpLevels) totals[threadIdx.x] = carry[threadIdx.x];
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    uint32_t s = 0;
+    for (int w = 0; w < kScanThreads / 32; ++w) s += sh[w];
+    return s;
 }
+
+__global__ void __launch_bounds__(kScanThreads) csf_scan_partials(const uint32_t *__restrict__ block_counts, int64_t nblocks,
+                                                                  uint32_t *__restrict__ partials) {
+    __shared__ uint32_t sh[kScanThreads / 32];
+    uint32_t mine[kCpLevels] = {0, 0, 0};
+    for (int k = 0; k < kScanPer; ++k) {
+        const int64_t b = (int64_t)blockIdx.x * kScanChunk + k * kScanThreads + threadIdx.x;
+        if (b < nblocks)
+#pragma unroll
+            for (int l = 0; l < kCpLevels; ++l) mine[l] += block_counts[b * kCpLevels + l];
+    }
+#pragma unroll
+    for (int l = 0; l < kCpLevels; ++l) {
+        const uint32_t s = block_sum(mine[l], sh);
+        if (threadIdx.x == 0) partials[(int64_t)blockIdx.x * kCpLevels + l] = s;
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads) csf_scan_apply(uint32_t *block_counts, int64_t nblocks,
+                                                               const uint32_t *__restrict__ partials, uint32_t *totals) {
+    __shared__ uint32_t sh[kScanThreads / 32];
+    __shared__ uint32_t wsum[kScanThreads / 32][kCpLevels];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // counts of kScanPer consecutive blocks per thread
+    uint32_t c[kScanPer][kCpLevels], mine[kCpLevels] = {0, 0, 0};
+    const int64_t b0 = (int64_t)blockIdx.x * kScanChunk + (int64_t)threadIdx.x * kScanPer;
+#pragma unroll
+    for (int k = 0; k < kScanPer; ++k)
+#pragma unroll
+        for (int l = 0; l < kCpLevels; ++l) {
+            c[k][l] = b0 + k < nblocks ? block_counts[(b0 + k) * kCpLevels + l] : 0;
+            mine[l] += c[k][l];
+        }
+#pragma unroll
+    for (int l = 0; l < kCpLevels; ++l) {
+        // sum of the chunks in front of this one
+        uint32_t before = 0;
+        for (int q = threadIdx.x; q < (int)blockIdx.x; q += kScanThreads) before += partials[(int64_t)q * kCpLevels + l];
+        before = block_sum(before, sh);
+        // exclusive scan of the threads' sums
+        uint32_t inc = mine[l];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        if (lane == 31) wsum[warp][l] = inc;
+        __syncthreads();
+        uint32_t run = before + inc - mine[l];
+        for (int w = 0; w < warp; ++w) run += wsum[w][l];
+#pragma unroll
+        for (int k = 0; k < kScanPer; ++k) {
+            if (b0 + k < nblocks) block_counts[(b0 + k) * kCpLevels + l] = run;
+            run += c[k][l];
+        }
+        if (b0 <= nblocks - 1 && nblocks - 1 < b0 + kScanPer) totals[l] = run;     // the thread that owns the last block
+    }
+}
+
+inline void launch_csf_scan(uint32_t *block_counts, int64_t nblocks, uint32_t *totals, cudaStream_t stream) {
+    const unsigned chunks = (unsigned)((nblocks + kScanChunk - 1) / kScanChunk);
+    uint32_t *partials = block_counts + nblocks * kCpLevels;        // behind the counts (see scan_partials_room)
+    CB_LAUNCH("csf_scan_partials", stream, csf_scan_partials<<<chunks, kScanThreads, 0, stream>>>(block_counts, nblocks, partials));
+    CB_LAUNCH("csf_scan_apply", stream, csf_scan_apply<<<chunks, kScanThreads, 0, stream>>>(block_counts, nblocks, partials, totals));
+}
+
+// numbers to allocate behind the per-block counts for the chunk sums of the scan
+inline int64_t scan_partials_room(int64_t nblocks) { return kCpLevels * ((nblocks + kScanChunk - 1) / kScanChunk + 1); }
 
 struct CsfArrays {
     int32_t *pos[kMaxOrder];
@@ -835,7 +878,7 @@ const_status_t sort_and_count(uint64_t *&keys, uint64_t *&keys_alt, const void *
     if (s != CONST_OK) return s;
     const int64_t cp_blocks = (nnz + kCpTile - 1) / kCpTile;
     CB_LAUNCH("csf_count", stream, csf_count<<<(unsigned)cp_blocks, kCpThreads, 0, stream>>>(keys, nnz, ls, block_counts, status));
-    CB_LAUNCH("csf_scan_blocks", stream, csf_scan_blocks<<<1, 1024, 0, stream>>>(block_counts, cp_blocks, totals));
+    launch_csf_scan(block_counts, cp_blocks, totals, stream);
     return CONST_OK;
 }
 
@@ -1023,7 +1066,8 @@ const_status_t csf_build_impl(int order, const int64_t *dims, int64_t nnz, const
             CB_CUDA(tmp.alloc(&vals_alt, vsize * (nnz + 4)));
             CB_CUDA(tmp.alloc((void **)&small, kSmallBytes));
             CB_CUDA(tmp.alloc((void **)&sb.tile_status, sizeof(unsigned long long) * std::max<int64_t>(ntiles, 1) * kRsMaxBins));
-            CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * kCpLevels * std::max<int64_t>(cp_blocks, 1)));
+            CB_CUDA(tmp.alloc((void **)&block_counts, sizeof(uint32_t) * (kCpLevels * std::max<int64_t>(cp_blocks, 1) +
+                                                                        scan_partials_room(cp_blocks))));
             CB_CUDA(cudaMemsetAsync(small, 0, kSmallBytes, stream));
             sb.hist = reinterpret_cast<uint32_t *>(small);
             sb.counters = reinterpret_cast<uint32_t *>(small + kHistBytes);
@@ -1106,7 +1150,7 @@ constexpr size_t kNaHistBytes = sizeof(uint32_t) * kMaxPasses * kRsMaxBins;
 constexpr size_t kNaOffSmall = kNaOffHist + kNaHistBytes;                 // pass counters, level totals, status word
 constexpr size_t kNaSmallBytes = 256;
 constexpr size_t kNaOffBlockCounts = kNaOffSmall + kNaSmallBytes;
-constexpr size_t kNaBytes = kNaOffBlockCounts + ((sizeof(uint32_t) * kCpLevels * kNaCpBlocks + 255) / 256) * 256;
+constexpr size_t kNaBytes = kNaOffBlockCounts + ((sizeof(uint32_t) * kCpLevels * (kNaCpBlocks + 2) + 255) / 256) * 256;
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress: it is not
 // a device address and must never be handed to a kernel or to cudaMemset as if it were one.
