@@ -281,6 +281,16 @@ const_status_t const_plan_set_tensor_stage(const_plan_t *plan, int enable);
  */
 const_status_t const_plan_set_generic_executor(const_plan_t *plan, int enable);
 
+/*
+ * What the generic executor will do for this plan (Sec. 4.2 loop structure, as compiled): one line per loop and
+ * per assignment -- which loop is spread over thread blocks, which CSF operand a loop walks ("walks B level 1"),
+ * which operands it looks up ("locates D level 1") or that it runs over a dense range, where a workspace is
+ * cleared and how many elements it has, and the private loops of every assignment.  Text protocol as for
+ * const_schedule_cin (buf may be NULL, *needed receives the length including the terminator, CONST_ERR_WORKSPACE
+ * when truncated).  CONST_ERR_UNSUPPORTED for a plan the generic executor cannot run.  Host only.
+ */
+const_status_t const_plan_describe(const const_plan_t *plan, char *buf, int64_t buf_len, int64_t *needed);
+
 /* Synchronise `stream` and return the device-side status word of the plan's last executions
  * (CONST_OK, or the first error a kernel recorded, e.g. CONST_ERR_TIMEOUT). */
 const_status_t const_last_device_status(const_plan_t *plan, void *stream);

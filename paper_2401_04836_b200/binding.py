@@ -84,6 +84,8 @@ def load_library():
     lib.const_last_device_status.argtypes = [vp, vp]
     lib.const_plan_set_tensor_stage.argtypes = [vp, i32]
     lib.const_plan_set_tensor_stage.restype = i32
+    lib.const_plan_describe.argtypes = [vp, ctypes.c_char_p, i64, pp(i64)]
+    lib.const_plan_describe.restype = i32
     lib.const_plan_set_generic_executor.argtypes = [vp, i32]
     lib.const_plan_set_generic_executor.restype = i32
     lib.const_destroy.argtypes = [vp]
@@ -381,6 +383,16 @@ def const_execute(plan: PlanHandle, operands: Dict[str, Union[CsfHandle, "object
 
 def const_plan_set_tensor_stage(plan: PlanHandle, enable: bool) -> None:
     _check(load_library().const_plan_set_tensor_stage(plan.ptr, 1 if enable else 0), "const_plan_set_tensor_stage")
+
+
+def const_plan_describe(plan: PlanHandle) -> str:
+    """Listing of what the generic executor does for this plan (loops, drivers, workspaces)."""
+    lib = load_library()
+    need = ctypes.c_int64()
+    _check(lib.const_plan_describe(plan.ptr, None, 0, ctypes.byref(need)), "const_plan_describe")
+    buf = ctypes.create_string_buffer(max(int(need.value), 1))
+    _check(lib.const_plan_describe(plan.ptr, buf, len(buf), ctypes.byref(need)), "const_plan_describe")
+    return buf.value.decode()
 
 
 def const_plan_set_generic_executor(plan: PlanHandle, enable: bool) -> None:

@@ -359,6 +359,21 @@ const_status_t const_plan_set_tensor_stage(const_plan_t *h, int enable) {
     return CONST_OK;
 }
 
+const_status_t const_plan_describe(const const_plan_t *h, char *buf, int64_t buf_len, int64_t *needed) {
+    const const_plan *p = as_plan(h);
+    if (!p) return CONST_ERR_INVALID_ARG;
+    if (!p->tree_ok) return CONST_ERR_UNSUPPORTED;
+    const std::string text = tree::describe(p->tree);
+    if (needed) *needed = (int64_t)text.size() + 1;
+    if (buf && buf_len > 0) {
+        const size_t n = std::min<size_t>(text.size(), (size_t)buf_len - 1);
+        std::memcpy(buf, text.data(), n);
+        buf[n] = 0;
+        if (n < text.size()) return CONST_ERR_WORKSPACE;
+    }
+    return CONST_OK;
+}
+
 const_status_t const_plan_set_generic_executor(const_plan_t *h, int enable) {
     const_plan *p = const_cast<const_plan *>(as_plan(h));
     if (!p) return CONST_ERR_INVALID_ARG;

@@ -91,8 +91,14 @@ struct Compiled {
     int result_slot = -1;
     std::vector<int> root_driver;                          // per program: sparse slot driving the root loop or -1
     std::vector<int64_t> root_extent;                      // per program: extent of the root index (dense root loop)
+    std::string index_names;                               // index id -> letter
+    std::vector<std::vector<std::string>> stmt_text;       // per program, per statement: the assignment as it stands in the tree
+    std::vector<std::vector<std::string>> ws_text;         // per program, per private workspace: its reduced reference
     std::string error;
 };
+
+// Human-readable listing of the compiled programs: how every loop iterates and what each entry does.
+std::string describe(const Compiled &c);
 
 // Compiles a parsed and checked schedule.  False (with `error` set) when it exceeds the fixed capacities.
 bool compile(const PlanDesc &desc, Compiled &out);

@@ -59,6 +59,8 @@ struct Compiler {
             for (char x : c.loops)
                 if (!idx_id.count(x)) { const int id = (int)idx_id.size(); idx_id[x] = id; }
         if ((int)idx_id.size() > kMaxIdx) return fail("too many iteration indices for the generic executor");
+        out.index_names.assign(idx_id.size(), '?');
+        for (auto &kv : idx_id) out.index_names[(size_t)kv.second] = kv.first;
         for (int c = 0; c < m; ++c) {
             producer[d.tree[c].out.name] = c;
             consumer[d.tree[c].lhs.name] = c;
@@ -216,7 +218,14 @@ struct Compiler {
         Program p{};
         int n_loops = 0, n_stmts = 0;
         std::map<int, int> ws_id;         // producing contraction -> workspace id of this program
+        std::vector<std::string> stmt_text, ws_text;
     };
+
+    static std::string show(const TensorRef &r) {
+        std::string t = r.name + "(";
+        for (size_t i = 0; i < r.idx.size(); ++i) { if (i) t += ", "; t.push_back(r.idx[i]); }
+        return t + ")";
+    }
 
     bool new_loop(Emit &e, const LoopNode &node, const std::vector<int> &stmts, const std::string &bound, int &id) {
         if (e.n_loops >= kMaxLoops) return fail("too many loops for the generic executor");
@@ -260,6 +269,8 @@ struct Compiler {
         if (s.out.kind == kRefPrivate) s.out.slot = (int8_t)e.ws_id.at(s.out.slot);
         if (s.lhs.kind == kRefPrivate) s.lhs.slot = (int8_t)e.ws_id.at(s.lhs.slot);
         if (s.rhs.kind == kRefPrivate) s.rhs.slot = (int8_t)e.ws_id.at(s.rhs.slot);
+        const Contraction &rk = tree.reduced[c];
+        e.stmt_text.push_back(show(rk.out) + " += " + show(rk.lhs) + " * " + show(rk.rhs));
         int at;
         return push(e, kOpStmt, e.n_stmts++, at);
     }
@@ -295,6 +306,7 @@ struct Compiler {
                 e.ws_id[c] = id;
                 const int64_t n = elems(tree.reduced[c].out.idx);
                 e.p.ws[id] = Workspace{e.p.block_scratch, n};
+                e.ws_text.push_back(show(tree.reduced[c].out));
                 e.p.block_scratch += (n + 1) / 2 * 2;           // keeps 16-byte alignment for fp64
             }
         driver = -1;
@@ -325,6 +337,8 @@ struct Compiler {
             root_extent = extent(root.index);
         }
         out.programs.push_back(e.p);
+        out.stmt_text.push_back(e.stmt_text);
+        out.ws_text.push_back(e.ws_text);
         return true;
     }
 
@@ -342,6 +356,43 @@ struct Compiler {
 };
 
 }  // namespace
+
+std::string describe(const Compiled &c) {
+    std::string text;
+    auto loop_text = [&](const Loop &L) {
+        std::string t(1, c.index_names[(size_t)L.index]);
+        if (L.driver >= 0) t += ": walks " + c.sparse_names[(size_t)L.driver] + " level " + std::to_string(L.level);
+        else t += ": dense range 0.." + std::to_string(L.extent);
+        for (int f = 0; f < L.n_follow; ++f)
+            t += std::string(f ? ", " : "; locates ") + c.sparse_names[(size_t)L.follow[f]] + " level " + std::to_string(L.flevel[f]);
+        return t;
+    };
+    for (size_t r = 0; r < c.programs.size(); ++r) {
+        const Program &p = c.programs[r];
+        text += "entry " + std::to_string(r) + ": ";
+        text += p.root_loop >= 0 ? "blocks over " + loop_text(p.loops[p.root_loop]) : std::string("one block");
+        text += "\n";
+        int depth = 1;
+        for (int pc = 0; pc < p.n_instr; ++pc) {
+            const Instr in = p.instr[pc];
+            if (in.op == kOpLoopEnd) { --depth; continue; }
+            text += std::string(2 * (size_t)depth, ' ');
+            if (in.op == kOpLoopBegin) {
+                text += "loop " + loop_text(p.loops[in.arg]) + "\n";
+                ++depth;
+            } else if (in.op == kOpZero) {
+                text += "zero " + c.ws_text[r][(size_t)in.arg] + " (" + std::to_string(p.ws[in.arg].size) + " elements per block)\n";
+            } else {
+                const Stmt &st = p.stmts[in.arg];
+                text += c.stmt_text[r][(size_t)in.arg];
+                for (int k = 0; k < st.n_priv; ++k)
+                    text += std::string(k ? ", " : "  [private loops: ") + loop_text(p.loops[st.priv[k]]);
+                text += st.n_priv ? "]\n" : "\n";
+            }
+        }
+    }
+    return text;
+}
 
 bool compile(const PlanDesc &desc, Compiled &out) {
     out = Compiled();

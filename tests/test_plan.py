@@ -164,3 +164,25 @@ def test_malformed_descriptors():
     ext = dict(w.extents); del ext["k"]
     assert bad(extents=ext) == 1
     assert bad(mode_orders={"Q": (0, 1, 2)}) == 1                              # unknown sparse tensor
+
+
+def test_generic_executor_program_of_the_running_example():
+    """How the compiled loop tree iterates (Sec. 4.2 structure; Fig. 5 schedule): r and j are fused and walk B, the
+    other CSF operands that carry them are looked up, X and Y are 2-D workspaces cleared per (r, j), and every
+    assignment keeps its own private loops in the order of its permutation."""
+    g, ext = _running_example()
+    p = cb.const_plan_create(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext, cb.F64)
+    lines = [l.strip() for l in cb.const_plan_describe(p).strip().split("\n")]
+    assert lines[0] == "entry 0: blocks over r: walks B level 0; locates C level 0, D level 0"
+    assert lines[1] == "loop j: walks B level 1; locates D level 1"
+    assert lines[2].startswith("zero X(i, q) (25 elements") and lines[3].startswith("zero Y(i, k) (25 elements")
+    assert lines[4].startswith("X(i, q) += A(i, p, q) * B(j, p, r)") and \
+        "p: walks B level 2; locates A level 0, q: walks A level 1, i: walks A level 2" in lines[4]
+    assert lines[5].startswith("Y(i, k) += X(i, q) * C(k, q, r)") and \
+        "q: walks C level 1, k: walks C level 2, i: dense range 0..5" in lines[5]
+    assert lines[6].startswith("R(i, j, k) += Y(i, k) * D(j, k, r)") and "k: walks D level 2, i: dense range 0..5" in lines[6]
+    assert len(lines) == 7
+    # unfused first contraction: X becomes a global workspace and the tree has two entries
+    p = cb.const_plan_create(g["expression"], g["tree"], g["mode_orders"], ["rjpqi", "irqkj", "irjk"], ext, cb.F64)
+    text = cb.const_plan_describe(p)
+    assert text.count("entry ") == 2 and "zero X" not in text and "zero Y(j, k)" in text
