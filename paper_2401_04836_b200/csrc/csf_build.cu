@@ -137,7 +137,6 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     uint64_t *keybuf = reinterpret_cast<uint64_t *>(smem_raw);
     V *valbuf = reinterpret_cast<V *>(smem_raw + kRsTile * sizeof(uint64_t));
     __shared__ uint32_t warp_hist[kRsWarps][kBins];
-    __shared__ uint32_t tile_hist[kBins];
     __shared__ uint32_t digit_excl[kBins];
     __shared__ uint32_t s_gbase[kBins];
     __shared__ uint32_t warp_tot[DPT][kRsWarps];
@@ -147,8 +146,6 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) { s_tile = atomicAdd(counter, 1u); s_abort = 0; }
     for (int x = threadIdx.x; x < kRsWarps * kBins; x += kRsThreads) (&warp_hist[0][0])[x] = 0;
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) tile_hist[q * kRsThreads + threadIdx.x] = 0;
     __syncthreads();
     const uint32_t tile = s_tile;
     const int64_t tile_base = (int64_t)tile * kRsTile;
@@ -179,18 +176,8 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
 
     // Digit counts of the tile first, so that later tiles can see them as early as possible:
     // the time from taking a tile to publishing its counts decides how long others wait.
-#pragma unroll
-    for (int i = 0; i < kRsItems; ++i) atomicAdd(&tile_hist[(unsigned)(key[i] >> shift) & kDigitMask], 1u);
-    __syncthreads();
     volatile unsigned long long *st = status;
     uint32_t count[DPT];
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        const int d = q * kRsThreads + threadIdx.x;
-        count[q] = tile_hist[d];
-        if (!withhold)      // (test hook: with the counts withheld, every later tile's bounded wait runs out)
-            st[(size_t)tile * kBins + d] = status_word(epoch, tile == 0 ? kFlagPrefix : kFlagOwn, count[q]);
-    }
 
     // Rank inside the warp: keys with equal digits keep their order (item, lane).  The lanes holding
     // another digit are collected from one ballot per digit bit (the match instruction costs one
@@ -228,6 +215,9 @@ __global__ void __launch_bounds__(kRsThreads, 3) rs_onesweep(const uint64_t *__r
             warp_hist[w][d] = run;
             run += c;
         }
+        count[q] = run;     // the tile's count of digit d: published now, so that later tiles can go on
+        if (!withhold)      // (test hook: with the counts withheld, every later tile's bounded wait runs out)
+            st[(size_t)tile * kBins + d] = status_word(epoch, tile == 0 ? kFlagPrefix : kFlagOwn, count[q]);
         incl[q] = count[q];
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
