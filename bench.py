@@ -41,7 +41,7 @@ ORACLE_SAMPLE_NNZ = {1: 20_000, 2: 20_000_000, 3: 3_000_000, 4: 40_000_000, 5: 2
 # summarised under profiles/; the kernels stream their inputs once, so the traffic of a full-size launch is this
 # figure times its nonzero count.  Only valid for the kernel version the capture was taken from: an entry is
 # dropped (traffic null) when its kernel changes.
-NCU_TRAFFIC_BYTES_PER_NNZ = {("ttmc3", "rs_onesweep"): 525.5e6 / 23.1e6, ("ttmc3", "chain3_kernel"): 236.3e6 / 23.1e6}
+NCU_TRAFFIC_BYTES_PER_NNZ = {("ttmc3", "rs_onesweep"): 527.0e6 / 23.1e6, ("ttmc3", "chain3_kernel"): 234.9e6 / 23.1e6}
 
 
 def measured_peaks():
