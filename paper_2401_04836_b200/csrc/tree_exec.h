@@ -61,6 +61,8 @@ struct Workspace { int64_t offset, size; };      // block-private: elements, off
 struct Program {
     int32_t n_instr;
     int32_t root_loop;             // loop spread over the blocks, -1: the entry is a bare assignment
+    int32_t root_loop2;            // >= 0: the loop below it, walking level 1 of the same operand, is spread over the
+                                   // blocks together with it: a block takes one level-1 node (two fused loops at once)
     int64_t block_scratch;         // elements of private workspace per block
     Instr instr[kMaxInstr];
     Loop loops[kMaxLoops];
@@ -78,7 +80,8 @@ struct SparsePtrs {
 struct Bindings {
     SparsePtrs sp[kMaxSparse];
     void *global[kMaxDense];       // dense inputs, the result, global workspaces
-    void *scratch;                 // private workspaces: block b owns [b * block_scratch, (b + 1) * block_scratch)
+    void *scratch;                 // private workspaces: block b owns [b * block_scratch, (b + 1) * block_scratch);
+                                   // NULL: they fit in the block's shared memory and live there
 };
 
 // What const_execute needs besides the programs.
@@ -90,6 +93,7 @@ struct Compiled {
     std::vector<bool> global_is_workspace;
     int result_slot = -1;
     std::vector<int> root_driver;                          // per program: sparse slot driving the root loop or -1
+    std::vector<bool> root_flattened;                      // per program: blocks take level-1 nodes of that operand
     std::vector<int64_t> root_extent;                      // per program: extent of the root index (dense root loop)
     std::string index_names;                               // index id -> letter
     std::vector<std::vector<std::string>> stmt_text;       // per program, per statement: the assignment as it stands in the tree

@@ -3,7 +3,9 @@
 // workspaces fused on r and j (Fig. 5), order-4 MTTKRP, TTMc at ranks the hand-written kernels do not
 // cover, the scatter form of the two-contraction network, or a network multiplied by a sparse 0/1 map
 // (Sec. 5.1, Eq. 2).  Slower than the hand-written families; it exists so that every schedule the checker
-// accepts can run.
+// accepts can run.  One iteration of the outermost fused loop (of the two outermost, when both walk the same
+// operand) goes to a block, or to a warp when its workspaces are small; the workspaces live in shared memory
+// when they fit there.
 #include <vector>
 
 #include "common.cuh"
@@ -92,21 +94,36 @@ __device__ __forceinline__ void update(const Stmt &s, const Program &p, const Bi
     atomicAdd(dst + address<T>(s.out, st), v);
 }
 
-// One assignment with its private loops: loop 0 over the warps (over all threads when it is the only one),
-// loop 1 over the lanes, deeper loops in sequence.
-template <typename T>
+// Who executes one iteration of the loops spread over the grid: a whole block, or (for small workspaces, where
+// the work of one iteration is small too) one warp of it, eight iterations in flight per block.
+template <bool WARP>
+struct Group {
+    static __device__ __forceinline__ int tid() { return WARP ? (int)(threadIdx.x & 31) : (int)threadIdx.x; }
+    static __device__ __forceinline__ int size() { return WARP ? 32 : (int)blockDim.x; }
+    static __device__ __forceinline__ int warp() { return WARP ? 0 : (int)(threadIdx.x >> 5); }
+    static __device__ __forceinline__ int warps() { return WARP ? 1 : (int)(blockDim.x >> 5); }
+    static __device__ __forceinline__ void sync() {
+        if (WARP) __syncwarp();
+        else __syncthreads();
+    }
+};
+
+// One assignment with its private loops: loop 0 over the warps of the group (over all its threads when it is
+// the only one), loop 1 over the lanes, deeper loops in sequence.
+template <typename T, bool WARP>
 __device__ void run_statement(const Stmt &s, const Program &p, const Bindings &b, State &st, T *scratch) {
+    using G = Group<WARP>;
     for (int k = 0; k < s.n_sparse; ++k)
-        if (st.absent[s.sparse[k]] != kAbsentNone) return;           // an operand has nothing here (uniform over the block)
+        if (st.absent[s.sparse[k]] != kAbsentNone) return;           // an operand has nothing here (uniform over the group)
     const int n = s.n_priv;
     if (n == 0) {
-        if (threadIdx.x == 0) update<T>(s, p, b, st, scratch);
+        if (G::tid() == 0) update<T>(s, p, b, st, scratch);
         return;
     }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31, warp = G::warp(), warps = G::warps();
     int32_t cur[kMaxPriv], end[kMaxPriv];
-    auto first = [&](int d) { return n == 1 ? (int)threadIdx.x : d == 0 ? warp : d == 1 ? lane : 0; };
-    auto step = [&](int d) { return n == 1 ? (int)blockDim.x : d == 0 ? warps : d == 1 ? 32 : 1; };
+    auto first = [&](int d) { return n == 1 ? G::tid() : d == 0 ? warp : d == 1 ? lane : 0; };
+    auto step = [&](int d) { return n == 1 ? G::size() : d == 0 ? warps : d == 1 ? 32 : 1; };
     int d = 0;
     loop_range(p.loops[s.priv[0]], b, st, cur[0], end[0]);
     cur[0] += first(0);
@@ -134,42 +151,82 @@ __device__ void run_statement(const Stmt &s, const Program &p, const Bindings &b
     for (int k = 0; k < s.n_sparse; ++k) st.absent[s.sparse[k]] = kAbsentNone;
 }
 
-template <typename T>
+// The instructions of one iteration of the loops spread over the grid.
+template <typename T, bool WARP>
+__device__ void run_body(const Program &p, const Bindings &b, State &st, T *scratch) {
+    using G = Group<WARP>;
+    int32_t cur[kMaxLoops], end[kMaxLoops];
+    int pc = 0;
+    while (pc < p.n_instr) {
+        const Instr in = p.instr[pc];
+        if (in.op == kOpZero) {
+            T *w = scratch + p.ws[in.arg].offset;
+            for (int64_t e = G::tid(); e < p.ws[in.arg].size; e += G::size()) w[e] = T(0);
+            G::sync();
+            ++pc;
+        } else if (in.op == kOpStmt) {
+            run_statement<T, WARP>(p.stmts[in.arg], p, b, st, scratch);
+            G::sync();
+            ++pc;
+        } else if (in.op == kOpLoopBegin) {
+            const Loop &L = p.loops[in.arg];
+            loop_range(L, b, st, cur[in.arg], end[in.arg]);
+            if (cur[in.arg] >= end[in.arg]) { pc = in.jump; continue; }
+            bind(L, b, st, cur[in.arg]);
+            ++pc;
+        } else {                                                  // kOpLoopEnd
+            if (++cur[in.arg] < end[in.arg]) {
+                bind(p.loops[in.arg], b, st, cur[in.arg]);
+                pc = in.jump;
+            } else {
+                ++pc;
+            }
+        }
+    }
+}
+
+// root_count: iterations of the loops spread over the grid (level-1 nodes of the driving operand when two
+// loops are spread together).  Groups take runs of `chunk` consecutive iterations, so that the level-0 node
+// above a level-1 node is searched for once per run and followed from there.
+// local_scratch: the private workspaces of a group live in shared memory (b.scratch is then unused).
+template <typename T, bool WARP>
 __global__ void __launch_bounds__(kThreads) tree_kernel(const __grid_constant__ Program p, const __grid_constant__ Bindings b,
-                                                        int64_t root_count) {
+                                                        int64_t root_count, int32_t chunk, int32_t local_scratch) {
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
     State st;
     for (int k = 0; k < kMaxSparse; ++k) st.absent[k] = kAbsentNone;
-    T *scratch = static_cast<T *>(b.scratch) + (int64_t)blockIdx.x * p.block_scratch;
-    int32_t cur[kMaxLoops], end[kMaxLoops];
+    const int groups_per_block = WARP ? (int)(blockDim.x >> 5) : 1;
+    const int group_in_block = WARP ? (int)(threadIdx.x >> 5) : 0;
+    const int64_t group = (int64_t)blockIdx.x * groups_per_block + group_in_block;
+    const int64_t groups = (int64_t)gridDim.x * groups_per_block;
+    T *scratch = local_scratch ? reinterpret_cast<T *>(dyn_smem) + (int64_t)group_in_block * p.block_scratch
+                               : static_cast<T *>(b.scratch) + group * p.block_scratch;
     const int64_t iterations = p.root_loop < 0 ? 1 : root_count;
-    for (int64_t it = blockIdx.x; it < iterations; it += gridDim.x) {
-        if (p.root_loop >= 0) bind(p.loops[p.root_loop], b, st, (int32_t)it);
-        int pc = 0;
-        while (pc < p.n_instr) {
-            const Instr in = p.instr[pc];
-            if (in.op == kOpZero) {
-                T *w = scratch + p.ws[in.arg].offset;
-                for (int64_t e = threadIdx.x; e < p.ws[in.arg].size; e += blockDim.x) w[e] = T(0);
-                __syncthreads();
-                ++pc;
-            } else if (in.op == kOpStmt) {
-                run_statement<T>(p.stmts[in.arg], p, b, st, scratch);
-                __syncthreads();
-                ++pc;
-            } else if (in.op == kOpLoopBegin) {
-                const Loop &L = p.loops[in.arg];
-                loop_range(L, b, st, cur[in.arg], end[in.arg]);
-                if (cur[in.arg] >= end[in.arg]) { pc = in.jump; continue; }
-                bind(L, b, st, cur[in.arg]);
-                ++pc;
-            } else {                                                  // kOpLoopEnd
-                if (++cur[in.arg] < end[in.arg]) {
-                    bind(p.loops[in.arg], b, st, cur[in.arg]);
-                    pc = in.jump;
+    for (int64_t run = group * chunk; run < iterations; run += groups * chunk) {
+        const int64_t run_end = run + chunk < iterations ? run + chunk : iterations;
+        int32_t above = -1;                                           // level-0 node over the current level-1 node
+        for (int64_t it = run; it < run_end; ++it) {
+            if (p.root_loop2 >= 0) {
+                const Loop &L0 = p.loops[p.root_loop];
+                const int32_t *pos1 = b.sp[L0.driver].pos[1];
+                int32_t at = above;
+                if (at < 0) {                                         // largest node whose children start at or before `it`
+                    int32_t lo = 0, hi = b.sp[L0.driver].n0 - 1;
+                    while (lo < hi) {
+                        const int32_t mid = lo + (hi - lo + 1) / 2;
+                        if ((int64_t)pos1[mid] <= it) lo = mid; else hi = mid - 1;
+                    }
+                    at = lo;
                 } else {
-                    ++pc;
+                    while ((int64_t)pos1[at + 1] <= it) ++at;         // ends: the last entry of pos1 is the node count
                 }
+                if (at != above) bind(L0, b, st, at);
+                above = at;
+                bind(p.loops[p.root_loop2], b, st, (int32_t)it);
+            } else if (p.root_loop >= 0) {
+                bind(p.loops[p.root_loop], b, st, (int32_t)it);
             }
+            run_body<T, WARP>(p, b, st, scratch);
         }
     }
 }
@@ -202,20 +259,45 @@ const_status_t run_tree(const tree::Compiled &cp, const_dtype_t dtype, const con
         CB_CUDA(cudaGetDevice(&dev));
         CB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     }
-    std::vector<int64_t> grids, counts;
+    // per program: who runs an iteration (block or warp), where its workspaces live, how the iterations are dealt out
+    constexpr int64_t kWarpScratchBytes = 4096;                       // up to here an iteration goes to one warp
+    constexpr int64_t kLocalScratchBytes = 96 * 1024;                 // up to here the workspaces live in shared memory
+    constexpr int kWarpsPerBlock = kThreads / 32;
+    struct Launch { int64_t grid, count; int chunk; bool warp, local; size_t smem; };
+    std::vector<Launch> launches;
     int64_t private_bytes = 0;
     for (size_t r = 0; r < cp.programs.size(); ++r) {
         const Program &p = cp.programs[r];
-        int64_t count = 1;
-        if (p.root_loop >= 0) count = cp.root_driver[r] >= 0 ? sparse[cp.root_driver[r]]->n[0] : cp.root_extent[r];
-        int64_t grid = std::max<int64_t>(1, std::min<int64_t>(count, (int64_t)sms * 8));
-        const int64_t per_block = p.block_scratch * (int64_t)esize;
-        if (per_block > kScratchBudget) return CONST_ERR_WORKSPACE;
-        if (per_block > 0) grid = std::min<int64_t>(grid, std::max<int64_t>(1, kScratchBudget / per_block));
-        grids.push_back(grid);
-        counts.push_back(count);
-        private_bytes = std::max<int64_t>(private_bytes, grid * per_block);
+        Launch L{};
+        L.count = 1;
+        if (p.root_loop >= 0) {
+            const int drv = cp.root_driver[r];
+            L.count = drv < 0 ? cp.root_extent[r] : sparse[drv]->n[p.root_loop2 >= 0 ? 1 : 0];
+        }
+        const int64_t per_group = p.block_scratch * (int64_t)esize;
+        if (per_group > kScratchBudget) return CONST_ERR_WORKSPACE;
+        L.warp = p.root_loop >= 0 && p.n_instr > 1 && per_group <= kWarpScratchBytes;
+        const int groups_per_block = L.warp ? kWarpsPerBlock : 1;
+        L.local = per_group * groups_per_block <= kLocalScratchBytes;
+        L.smem = L.local ? (size_t)(per_group * groups_per_block) : 0;
+        L.grid = std::max<int64_t>(1, std::min<int64_t>((L.count + groups_per_block - 1) / groups_per_block, (int64_t)sms * 8));
+        if (!L.local) {
+            L.grid = std::min<int64_t>(L.grid, std::max<int64_t>(1, kScratchBudget / per_group));
+            private_bytes = std::max<int64_t>(private_bytes, L.grid * per_group);
+        }
+        // runs of consecutive iterations per group: long enough to amortise the search for the node above,
+        // short enough to leave every group several runs
+        L.chunk = (int)std::max<int64_t>(1, std::min<int64_t>(32, L.count / (L.grid * groups_per_block * 8)));
+        launches.push_back(L);
     }
+    static PerDeviceOnce smem_once;
+    CB_CUDA(once_per_device(smem_once, [] {
+        cudaError_t e = cudaFuncSetAttribute(tree_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLocalScratchBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLocalScratchBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<double, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLocalScratchBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<double, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLocalScratchBytes);
+        return e;
+    }));
     const int64_t total_bytes = shared_elems * (int64_t)esize + private_bytes + 256;
     unsigned char *scratch = nullptr;
     CB_CUDA(cudaMallocAsync((void **)&scratch, (size_t)total_bytes, stream));
@@ -235,12 +317,19 @@ const_status_t run_tree(const tree::Compiled &cp, const_dtype_t dtype, const con
     if (e == cudaSuccess)                                             // "R[*] = 0" precedes the nest
         e = cudaMemsetAsync(out_dev, 0, (size_t)cp.global_elems[(size_t)cp.result_slot] * esize, stream);
     for (size_t r = 0; r < cp.programs.size() && e == cudaSuccess; ++r) {
-        if (counts[r] == 0) continue;
+        const Launch &L = launches[r];
+        if (L.count == 0) continue;
+        const unsigned grid = (unsigned)L.grid;
+        const int32_t local = L.local ? 1 : 0;
         CB_LAUNCH("tree_kernel", stream, {
-            if (dtype == CONST_F32)
-                tree_kernel<float><<<(unsigned)grids[r], kThreads, 0, stream>>>(cp.programs[r], b, counts[r]);
+            if (dtype == CONST_F32 && L.warp)
+                tree_kernel<float, true><<<grid, kThreads, L.smem, stream>>>(cp.programs[r], b, L.count, L.chunk, local);
+            else if (dtype == CONST_F32)
+                tree_kernel<float, false><<<grid, kThreads, L.smem, stream>>>(cp.programs[r], b, L.count, L.chunk, local);
+            else if (L.warp)
+                tree_kernel<double, true><<<grid, kThreads, L.smem, stream>>>(cp.programs[r], b, L.count, L.chunk, local);
             else
-                tree_kernel<double><<<(unsigned)grids[r], kThreads, 0, stream>>>(cp.programs[r], b, counts[r]);
+                tree_kernel<double, false><<<grid, kThreads, L.smem, stream>>>(cp.programs[r], b, L.count, L.chunk, local);
         });
         e = cudaGetLastError();
     }

@@ -312,6 +312,7 @@ struct Compiler {
         driver = -1;
         root_extent = 1;
         e.p.root_loop = -1;
+        e.p.root_loop2 = -1;
         if (!root.is_loop) {
             if (!emit_statement(e, root.contraction, {}, "")) return false;
         } else if (stmts.size() == 1) {
@@ -328,15 +329,38 @@ struct Compiler {
             int id;
             if (!new_loop(e, root, stmts, "", id)) return false;
             e.p.root_loop = id;
-            if (!emit_zeros(e, &root)) return false;
-            for (const LoopNode &c : root.body)
-                if (!emit_node(e, c, std::string(1, root.index))) return false;
+            // Two fused loops at once: when the body of the outermost loop is nothing but the next fused loop, and
+            // both walk consecutive levels of the same CSF operand, a block takes one level-1 node of that operand
+            // (a pair of coordinates) instead of a whole level-0 node: far more blocks, far more evenly loaded.
+            const LoopNode *inner = root.body.size() == 1 && root.body[0].is_loop ? &root.body[0] : nullptr;
+            std::vector<int> inner_stmts;
+            if (inner) count_statements(*inner, inner_stmts);
+            bool flattened = false;
+            if (inner && inner_stmts.size() >= 2 && !zero_at.count(&root) && e.p.loops[id].driver >= 0) {
+                int id2;
+                if (!new_loop(e, *inner, inner_stmts, std::string(1, root.index), id2)) return false;
+                if (e.p.loops[id2].driver == e.p.loops[id].driver && e.p.loops[id2].level == 1) {
+                    e.p.root_loop2 = id2;
+                    if (!emit_zeros(e, inner)) return false;
+                    for (const LoopNode &c : inner->body)
+                        if (!emit_node(e, c, std::string(1, root.index) + inner->index)) return false;
+                    flattened = true;
+                } else {
+                    --e.n_loops;                                  // not the same operand: the inner loop stays a uniform loop
+                }
+            }
+            if (!flattened) {
+                if (!emit_zeros(e, &root)) return false;
+                for (const LoopNode &c : root.body)
+                    if (!emit_node(e, c, std::string(1, root.index))) return false;
+            }
         }
         if (e.p.root_loop >= 0) {
             driver = e.p.loops[e.p.root_loop].driver;
             root_extent = extent(root.index);
         }
         out.programs.push_back(e.p);
+        out.root_flattened.push_back(e.p.root_loop2 >= 0);
         out.stmt_text.push_back(e.stmt_text);
         out.ws_text.push_back(e.ws_text);
         return true;
@@ -371,6 +395,7 @@ std::string describe(const Compiled &c) {
         const Program &p = c.programs[r];
         text += "entry " + std::to_string(r) + ": ";
         text += p.root_loop >= 0 ? "blocks over " + loop_text(p.loops[p.root_loop]) : std::string("one block");
+        if (p.root_loop2 >= 0) text += " | and over " + loop_text(p.loops[p.root_loop2]);
         text += "\n";
         int depth = 1;
         for (int pc = 0; pc < p.n_instr; ++pc) {
@@ -381,7 +406,7 @@ std::string describe(const Compiled &c) {
                 text += "loop " + loop_text(p.loops[in.arg]) + "\n";
                 ++depth;
             } else if (in.op == kOpZero) {
-                text += "zero " + c.ws_text[r][(size_t)in.arg] + " (" + std::to_string(p.ws[in.arg].size) + " elements per block)\n";
+                text += "zero " + c.ws_text[r][(size_t)in.arg] + " (" + std::to_string(p.ws[in.arg].size) + " elements per iteration in flight)\n";
             } else {
                 const Stmt &st = p.stmts[in.arg];
                 text += c.stmt_text[r][(size_t)in.arg];

@@ -173,15 +173,21 @@ def test_generic_executor_program_of_the_running_example():
     g, ext = _running_example()
     p = cb.const_plan_create(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext, cb.F64)
     lines = [l.strip() for l in cb.const_plan_describe(p).strip().split("\n")]
-    assert lines[0] == "entry 0: blocks over r: walks B level 0; locates C level 0, D level 0"
-    assert lines[1] == "loop j: walks B level 1; locates D level 1"
-    assert lines[2].startswith("zero X(i, q) (25 elements") and lines[3].startswith("zero Y(i, k) (25 elements")
-    assert lines[4].startswith("X(i, q) += A(i, p, q) * B(j, p, r)") and \
-        "p: walks B level 2; locates A level 0, q: walks A level 1, i: walks A level 2" in lines[4]
-    assert lines[5].startswith("Y(i, k) += X(i, q) * C(k, q, r)") and \
-        "q: walks C level 1, k: walks C level 2, i: dense range 0..5" in lines[5]
-    assert lines[6].startswith("R(i, j, k) += Y(i, k) * D(j, k, r)") and "k: walks D level 2, i: dense range 0..5" in lines[6]
-    assert len(lines) == 7
+    # both fused loops walk B, so the (r, j) pairs -- B's level-1 nodes -- are what the grid is spread over
+    assert lines[0] == ("entry 0: blocks over r: walks B level 0; locates C level 0, D level 0"
+                        " | and over j: walks B level 1; locates D level 1")
+    assert lines[1].startswith("zero X(i, q) (25 elements") and lines[2].startswith("zero Y(i, k) (25 elements")
+    assert lines[3].startswith("X(i, q) += A(i, p, q) * B(j, p, r)") and \
+        "p: walks B level 2; locates A level 0, q: walks A level 1, i: walks A level 2" in lines[3]
+    assert lines[4].startswith("Y(i, k) += X(i, q) * C(k, q, r)") and \
+        "q: walks C level 1, k: walks C level 2, i: dense range 0..5" in lines[4]
+    assert lines[5].startswith("R(i, j, k) += Y(i, k) * D(j, k, r)") and "k: walks D level 2, i: dense range 0..5" in lines[5]
+    assert len(lines) == 6
+    # the same holds for a TTMc at a rank the hand-written kernels do not cover: the (i, j) fibres of X are spread
+    p2 = cb.const_plan_create("Y[i,a,b] = X[i,j,k] * U[j,a] * V[k,b]",
+                              ["T[i,j,b] = X[i,j,k] * V[k,b]", "Y[i,a,b] = T[i,j,b] * U[j,a]"],
+                              {"X": (0, 1, 2)}, ["ijkb", "ijab"], {"i": 40, "j": 30, "k": 20, "a": 12, "b": 12}, cb.F64)
+    assert cb.const_plan_family(p2) == "tree" and " | and over j: walks X level 1" in cb.const_plan_describe(p2)
     # unfused first contraction: X becomes a global workspace and the tree has two entries
     p = cb.const_plan_create(g["expression"], g["tree"], g["mode_orders"], ["rjpqi", "irqkj", "irjk"], ext, cb.F64)
     text = cb.const_plan_describe(p)
