@@ -50,6 +50,8 @@ struct Stmt {
     int8_t priv[kMaxPriv];         // loop ids
     int8_t n_sparse;
     int8_t sparse[2];              // sparse slots it reads
+    int8_t fuse_tail;              // the innermost private loop is a plain dense range and the one around it locates no
+                                   // operand: the pair is dealt to the threads as one loop over their combined range
     Ref out, lhs, rhs;
 };
 

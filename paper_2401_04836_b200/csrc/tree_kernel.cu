@@ -109,7 +109,8 @@ struct Group {
 };
 
 // One assignment with its private loops: loop 0 over the warps of the group (over all its threads when it is
-// the only one), loop 1 over the lanes, deeper loops in sequence.
+// the only one), loop 1 over the lanes, deeper loops in sequence.  A dense innermost loop is first merged
+// with the loop around it (Stmt::fuse_tail), so that short sparse ranges still fill the lanes.
 template <typename T, bool WARP>
 __device__ void run_statement(const Stmt &s, const Program &p, const Bindings &b, State &st, T *scratch) {
     using G = Group<WARP>;
@@ -121,30 +122,51 @@ __device__ void run_statement(const Stmt &s, const Program &p, const Bindings &b
         return;
     }
     const int lane = threadIdx.x & 31, warp = G::warp(), warps = G::warps();
+    // m loops as they are dealt out: with fuse_tail the two innermost count as one, over (outer range) x (inner extent)
+    const bool fuse = s.fuse_tail != 0;
+    const int m = fuse ? n - 1 : n;
+    const int32_t inner_extent = fuse ? p.loops[s.priv[n - 1]].extent : 1;
+    int32_t fused_lo = 0;
     int32_t cur[kMaxPriv], end[kMaxPriv];
-    auto first = [&](int d) { return n == 1 ? G::tid() : d == 0 ? warp : d == 1 ? lane : 0; };
-    auto step = [&](int d) { return n == 1 ? G::size() : d == 0 ? warps : d == 1 ? 32 : 1; };
+    auto first = [&](int d) { return m == 1 ? G::tid() : d == 0 ? warp : d == 1 ? lane : 0; };
+    auto step = [&](int d) { return m == 1 ? G::size() : d == 0 ? warps : d == 1 ? 32 : 1; };
+    auto open = [&](int d) {                                        // range of dealt loop d under the current bindings
+        int32_t lo, hi;
+        loop_range(p.loops[s.priv[d]], b, st, lo, hi);
+        if (fuse && d == m - 1) {
+            fused_lo = lo;
+            cur[d] = first(d);
+            end[d] = (hi - lo) * inner_extent;
+        } else {
+            cur[d] = lo + first(d);
+            end[d] = hi;
+        }
+    };
     int d = 0;
-    loop_range(p.loops[s.priv[0]], b, st, cur[0], end[0]);
-    cur[0] += first(0);
+    open(0);
     while (d >= 0) {
         if (cur[d] >= end[d]) {
             --d;
             if (d >= 0) cur[d] += step(d);
             continue;
         }
-        const Loop &L = p.loops[s.priv[d]];
-        if (!bind(L, b, st, cur[d])) {                                // an operand of this assignment is absent
+        bool here;
+        if (fuse && d == m - 1) {
+            here = bind(p.loops[s.priv[d]], b, st, fused_lo + cur[d] / inner_extent);
+            bind(p.loops[s.priv[n - 1]], b, st, cur[d] % inner_extent);
+        } else {
+            here = bind(p.loops[s.priv[d]], b, st, cur[d]);
+        }
+        if (!here) {                                                  // an operand of this assignment is absent
             cur[d] += step(d);
             continue;
         }
-        if (d == n - 1) {
+        if (d == m - 1) {
             update<T>(s, p, b, st, scratch);
             cur[d] += step(d);
         } else {
             ++d;
-            loop_range(p.loops[s.priv[d]], b, st, cur[d], end[d]);
-            cur[d] += first(d);
+            open(d);
         }
     }
     // what the private loops bound is dead now; the operands stand where the uniform loops left them

@@ -262,6 +262,11 @@ struct Compiler {
             s.priv[s.n_priv++] = (int8_t)id;
             bound.push_back(n->index);
         }
+        if (s.n_priv >= 2) {
+            const Loop &inner = e.p.loops[s.priv[s.n_priv - 1]], &outer = e.p.loops[s.priv[s.n_priv - 2]];
+            s.fuse_tail = inner.driver < 0 && inner.n_follow == 0 && outer.n_follow == 0 &&
+                          (int64_t)inner.extent * outer.extent < (1ll << 31);
+        }
         const Contraction &k = d.tree[c];
         if (!make_ref(k.out, e.p, s.out) || !make_ref(k.lhs, e.p, s.lhs) || !make_ref(k.rhs, e.p, s.rhs)) return false;
         for (const Ref *r : {&s.lhs, &s.rhs})
