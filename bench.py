@@ -453,7 +453,7 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
                                            "frac": None, "traffic": None}
     fused = next((rooflines[k] for k in rooflines if k in FUSED_KERNELS and rooflines[k]), None)
 
-    # ---- CPU baseline (the oracle on a bounded sample, on this machine's host cores) and the run's own parity check ----
+    # ---- CPU baseline (the oracle on a bounded sample, on the host's cores) and the run's own parity check ----
     cpu_baseline, max_err_ratio = None, None
     if want_oracle:
         cpu_baseline, _, rows, S, A = time_oracle(w, args.oracle_nnz or ORACLE_SAMPLE_NNZ[config_id])
