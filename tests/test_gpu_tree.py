@@ -200,3 +200,38 @@ def test_empty_operand_and_operand_checks():
         cb.const_execute(plan, {"X": build_csf(w.sparse["X"], (0, 1, 2)), "U": to_dev(w.dense["U"])}, out)
     with pytest.raises(cb.ConstError):
         cb.const_plan_set_generic_executor(plan, False)                  # this plan has no other kernel
+
+
+def test_random_legal_schedules_of_the_running_example():
+    """Sixty seeded schedules of R_ijk = A_ipq B_jpr C_kqr D_jkr: random loop permutations per contraction (half of
+    them forced to share leading loops, so that fused nests with reduced workspaces come up as often as plain
+    ones), every CSF operand stored in the mode order its reader's loops ask for (Sec. 3.2).  Whatever the checker
+    accepts must run and give the one result the expression defines."""
+    rng = np.random.default_rng(2401)
+    ext = {"i": 6, "j": 7, "k": 5, "p": 6, "q": 4, "r": 5}
+    shape = {"A": "ipq", "B": "jpr", "C": "kqr", "D": "jkr"}
+    reader = {"A": 0, "B": 0, "C": 1, "D": 2}
+    sparse = {t: sparse_input(rng, tuple(ext[x] for x in idx), 70, np.float64) for t, idx in shape.items()}
+    expr = "R[i,j,k] = A[i,p,q] * B[j,p,r] * C[k,q,r] * D[j,k,r]"
+    tree = ["X[i,j,q,r] = A[i,p,q] * B[j,p,r]", "Y[i,j,k,r] = X[i,j,q,r] * C[k,q,r]", "R[i,j,k] = Y[i,j,k,r] * D[j,k,r]"]
+    S, A = oc.nary_einsum(expr, {t: coo(op) for t, op in sparse.items()}, ext)
+    ran, fused = 0, 0
+    for trial in range(60):
+        loops = []
+        lead = "".join(rng.permutation(list("ijr")))[: int(rng.integers(1, 4))] if trial % 2 else ""
+        for idx in ("ijpqr", "ijkqr", "ijkr"):
+            rest = [c for c in idx if c not in lead]
+            loops.append(lead + "".join(rng.permutation(rest)))
+        mo = {n: [int(x) for x in np.argsort([loops[reader[n]].index(c) for c in shape[n]])] for n in shape}
+        try:
+            plan = cb.const_plan_create(expr, tree, mo, loops, ext, cb.F64)
+        except cb.ConstError as e:
+            assert e.status == 3, (loops, e.status)              # an illegal schedule is the only reason to refuse
+            continue
+        text = cb.const_plan_describe(plan)
+        fused += "zero " in text
+        out, family = run_tree(expr, tree, mo, loops, ext, cb.F64, sparse, {}, (6, 7, 5))
+        assert family == "tree"
+        assert_close(out, S, A, np.float64)
+        ran += 1
+    assert ran >= 40 and fused >= 10, (ran, fused)
