@@ -235,3 +235,34 @@ def test_random_legal_schedules_of_the_running_example():
         assert_close(out, S, A, np.float64)
         ran += 1
     assert ran >= 40 and fused >= 10, (ran, fused)
+
+
+@pytest.mark.parametrize("dtype", [cb.F64, cb.F32])
+def test_every_tree_of_the_network_under_random_schedules(dtype):
+    """Z_im = U_ijk V_jl W_klm (Sec. 1) through each of its three contraction trees -- (U V) W, U (V W) and
+    (U W) V -- with ninety seeded loop orders, half of them sharing leading loops so that the intermediate loses
+    modes.  All trees and all schedules define the same Z."""
+    rng = np.random.default_rng(4836)
+    ext = {"i": 9, "j": 7, "k": 8, "l": 5, "m": 6}
+    shape = {"U": "ijk", "W": "klm"}
+    sparse = {t: sparse_input(rng, tuple(ext[x] for x in idx), 90, NP[dtype]) for t, idx in shape.items()}
+    V = rng.uniform(-1.0, 1.0, (ext["j"], ext["l"])).astype(NP[dtype])
+    expr = "Z[i,m] = U[i,j,k] * V[j,l] * W[k,l,m]"
+    trees = [(["T[i,k,l] = U[i,j,k] * V[j,l]", "Z[i,m] = T[i,k,l] * W[k,l,m]"], ("ijkl", "iklm"), {"U": 0, "W": 1}),
+             (["T[j,k,m] = V[j,l] * W[k,l,m]", "Z[i,m] = U[i,j,k] * T[j,k,m]"], ("jklm", "ijkm"), {"U": 1, "W": 0}),
+             (["T[i,j,l,m] = U[i,j,k] * W[k,l,m]", "Z[i,m] = T[i,j,l,m] * V[j,l]"], ("ijklm", "ijlm"), {"U": 0, "W": 0})]
+    ops = {t: coo(op) for t, op in sparse.items()}
+    ops["V"] = V
+    S, A = oc.nary_einsum(expr, ops, ext)
+    fused = 0
+    for trial in range(90):
+        tree, idxs, reader = trees[trial % 3]
+        shared = [c for c in idxs[0] if c in idxs[1]]
+        lead = "".join(rng.permutation(shared))[: int(rng.integers(0, len(shared) + 1))] if trial % 2 else ""
+        loops = [lead + "".join(rng.permutation([c for c in s if c not in lead])) for s in idxs]
+        mo = {n: [int(x) for x in np.argsort([loops[reader[n]].index(c) for c in shape[n]])] for n in shape}
+        plan = cb.const_plan_create(expr, tree, mo, loops, ext, dtype)
+        fused += "zero " in cb.const_plan_describe(plan)
+        out, _ = run_tree(expr, tree, mo, loops, ext, dtype, sparse, {"V": V}, (ext["i"], ext["m"]), generic=True)
+        assert_close(out, S, A, NP[dtype])
+    assert fused >= 20, fused
