@@ -266,3 +266,33 @@ def test_every_tree_of_the_network_under_random_schedules(dtype):
         out, _ = run_tree(expr, tree, mo, loops, ext, dtype, sparse, {"V": V}, (ext["i"], ext["m"]), generic=True)
         assert_close(out, S, A, NP[dtype])
     assert fused >= 20, fused
+
+
+def test_medium_sizes_reach_every_way_the_iterations_are_dealt_out():
+    """Sizes at which the executor's launch logic leaves its small-case settings: (a) 400 K nonzeros in about as
+    many (i, j) fibres with a 12-element workspace -- one fibre per warp, runs of several consecutive fibres per
+    warp, the slice above a fibre followed along the run; (b) fp64 workspaces of 4.8 KB -- one fibre per block,
+    workspaces in shared memory; (c) a 122 KB workspace per outer iteration -- workspaces in global scratch."""
+    w = ttmc3_workload((4000, 300, 400), 400_000, (12, 12), slice_s=1.1, value="pm1", config_id=61)
+    S, A = oracle(w)
+    out, family = run_tree(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, cb.F32, w.sparse, w.dense,
+                           w.out_shape)
+    assert family == "tree"
+    assert_close(out, S, A, np.float32)
+
+    w = ttmc4_workload((300, 100, 20, 20), 60_000, 24, slice_s=1.0, value="pm1", config_id=62)
+    X = w.sparse["X"]
+    sparse = {"X": gen.SparseOperand(X.coords, X.vals.astype(np.float64), X.dims)}
+    dense = {n: a.astype(np.float64) for n, a in w.dense.items()}
+    S, A = oracle(w)                                              # fp64 throughout; the inputs are fp32 values
+    out, family = run_tree(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, cb.F64, sparse, dense,
+                           w.out_shape)
+    assert family == "tree"
+    assert_close(out, S, A, np.float64)
+
+    w = network_workload(160, 96, 8, 0.3, config_id=63)
+    S, A = oracle(w)
+    out, family = run_tree(w.expression, w.tree, {"U": (0, 1, 2), "W": (0, 1, 2)}, ["ijkl", "iklm"], w.extents, cb.F64,
+                           w.sparse, w.dense, w.out_shape)
+    assert family == "tree"
+    assert_close(out, S, A, np.float64)
