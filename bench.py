@@ -353,6 +353,17 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
     gc.disable()
     t_begin = time.monotonic()
     total_ms, per_step, per_exec = timed_loop()
+    remeasured = None
+    if max(per_step) > 3.0 * float(np.median(per_step)) and total_ms / steps > 1.2 * float(np.median(per_step)):
+        # One step far outside the others (seen on shared hosts: a stall of the launching thread of a second or
+        # so while the kernels themselves keep their times) spoils the mean.  Like a run with a throttled clock
+        # it is measured again, once, and the first attempt is reported next to the second.
+        remeasured = {"first_ms_per_step": total_ms / steps, "first_step_ms_max": float(max(per_step)),
+                      "first_step_ms_median": float(np.median(per_step)),
+                      "why": "one step above 3x the median step time; measured again once"}
+        cb.const_profile_enable(True)                    # also clears the records of the first attempt
+        t_begin = time.monotonic()
+        total_ms, per_step, per_exec = timed_loop()
     t_end = time.monotonic()
     gc.enable()
     prof = cb.const_profile_read()
@@ -467,6 +478,7 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
     return {
         "workload": w.name, "dtype": "f32" if dtype == cb.F32 else "f64",
         "ms_per_step": ms_per_step, "step_ms_median": float(np.median(per_step)), "step_ms_min": float(np.min(per_step)),
+        "remeasured": remeasured,
         "value": total_flops / (ms_per_step * 1e-3) / 1e9, "unit": "GFLOP/s",
         "nnz": nnz_total, "level_sizes": level_sizes, "bins": bins,
         "l2": "inputs larger than L2 (no flush)" if not fits_l2 else
@@ -605,7 +617,7 @@ def main():
                    "wall_s": round(setup_s, 1),
                    "per_config": {str(cid): brief(results[cid]) for cid in sorted(results)}},
         "stages": h["stages"], "hbm_gbs": h["hbm_gbs"],
-        "step_ms_median": h["step_ms_median"], "step_ms_min": h["step_ms_min"],
+        "step_ms_median": h["step_ms_median"], "step_ms_min": h["step_ms_min"], "remeasured": h["remeasured"],
         "kernels": h["kernels"], "roofline": h["roofline"], "roofline_fused_kernel": h["roofline_fused_kernel"],
         "rooflines": h["rooflines"], "gather_ceiling": h["gather_ceiling"],
         "cpu_baseline": h["cpu_baseline"], "max_err_ratio": h["max_err_ratio"], "e2e": h["e2e"],
