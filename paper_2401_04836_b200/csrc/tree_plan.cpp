@@ -417,7 +417,7 @@ std::string describe(const Compiled &c) {
                 text += c.stmt_text[r][(size_t)in.arg];
                 for (int k = 0; k < st.n_priv; ++k)
                     text += std::string(k ? ", " : "  [private loops: ") + loop_text(p.loops[st.priv[k]]);
-                text += st.n_priv ? "]\n" : "\n";
+                text += st.n_priv ? (st.fuse_tail ? "; last two dealt out as one]\n" : "]\n") : "\n";
             }
         }
     }

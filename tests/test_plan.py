@@ -183,6 +183,10 @@ def test_generic_executor_program_of_the_running_example():
         "q: walks C level 1, k: walks C level 2, i: dense range 0..5" in lines[4]
     assert lines[5].startswith("R(i, j, k) += Y(i, k) * D(j, k, r)") and "k: walks D level 2, i: dense range 0..5" in lines[5]
     assert len(lines) == 6
+    # a dense innermost loop is dealt to the threads together with the loop around it, unless that loop has to
+    # locate an operand (p locates A, so the first assignment keeps its three loops apart)
+    assert lines[4].endswith("last two dealt out as one]") and lines[5].endswith("last two dealt out as one]")
+    assert lines[3].endswith("i: walks A level 2]")
     # the same holds for a TTMc at a rank the hand-written kernels do not cover: the (i, j) fibres of X are spread
     p2 = cb.const_plan_create("Y[i,a,b] = X[i,j,k] * U[j,a] * V[k,b]",
                               ["T[i,j,b] = X[i,j,k] * V[k,b]", "Y[i,a,b] = T[i,j,b] * U[j,a]"],
