@@ -252,6 +252,8 @@ def measure_config(cb, torch, w, config_id, args, peaks, hbm_peak, peak_kind, ra
     plan = cb.const_plan_create(w.expression, w.tree, w.mode_orders, w.loop_orders, w.extents, dtype)
     if args.tensor_stage >= 0 and w.family in ("ttmc4", "ttmc3"):
         cb.const_plan_set_tensor_stage(plan, bool(args.tensor_stage))
+    if args.generic_executor:
+        cb.const_plan_set_generic_executor(plan, True)
     stream = torch.cuda.current_stream()
     bins_override = tuple(int(x) for x in args.bins.split(",")) if args.bins else None
 
@@ -509,6 +511,8 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--impl", default="const")
     ap.add_argument("--oracle-nnz", type=int, default=0, help="nonzeros in the CPU-baseline sample (0 = auto)")
+    ap.add_argument("--generic-executor", action="store_true",
+                    help="run the schedules on the generic loop-tree executor instead of the hand-written kernels")
     ap.add_argument("--tensor-stage", type=int, default=-1,
                     help="TTMc: 1 = dense per-slice stage on the tensor cores, 0 = on the FMA pipes, -1 = library default")
     ap.add_argument("--bins", default="", help="light_max,heavy_max,chunk nonzero thresholds of the load balancer (default: the library's)")
