@@ -53,6 +53,16 @@ struct Stmt {
     int8_t fuse_tail;              // the innermost private loop is a plain dense range and the one around it locates no
                                    // operand: the pair is dealt to the threads as one loop over their combined range
     Ref out, lhs, rhs;
+    // Strength reduction of the innermost dealt loop (the last private loop, or the last two when fuse_tail):
+    // when neither of them locates an operand (`fast`), the element a reference touches there is
+    //   base + coordinate_A * sA + coordinate_B * sB + position_A * pA + position_B * pB
+    // with A the outer and B the inner of the two (A unused without fuse_tail), `base` taken once per entry into
+    // the loop, coordinate = the index value, position = the place in the driving operand's level.  Dense
+    // references use sA / sB (their strides for the two indices), a sparse reference whose leaf level one of the
+    // two loops walks uses pA / pB = 1, any other sparse reference is a constant of the loop.
+    int8_t fast;
+    int32_t sA[3], sB[3];          // out, lhs, rhs
+    int8_t pA[3], pB[3];
 };
 
 enum Op : int8_t { kOpLoopBegin = 0, kOpLoopEnd = 1, kOpZero = 2, kOpStmt = 3 };

@@ -126,47 +126,100 @@ __device__ void run_statement(const Stmt &s, const Program &p, const Bindings &b
     const bool fuse = s.fuse_tail != 0;
     const int m = fuse ? n - 1 : n;
     const int32_t inner_extent = fuse ? p.loops[s.priv[n - 1]].extent : 1;
-    int32_t fused_lo = 0;
     int32_t cur[kMaxPriv], end[kMaxPriv];
     auto first = [&](int d) { return m == 1 ? G::tid() : d == 0 ? warp : d == 1 ? lane : 0; };
     auto step = [&](int d) { return m == 1 ? G::size() : d == 0 ? warps : d == 1 ? 32 : 1; };
-    auto open = [&](int d) {                                        // range of dealt loop d under the current bindings
+    auto open = [&](int d) {                                        // range of dealt loop d (not the innermost) under the current bindings
+        loop_range(p.loops[s.priv[d]], b, st, cur[d], end[d]);
+        cur[d] += first(d);
+    };
+    // ---- the innermost dealt loop, entered with every loop around it bound
+    auto innermost = [&]() {
+        const int dl = m - 1;
+        const Loop &LB = p.loops[s.priv[n - 1]];
+        const Loop &LA = p.loops[s.priv[fuse ? n - 2 : n - 1]];           // the loop whose range is walked
         int32_t lo, hi;
-        loop_range(p.loops[s.priv[d]], b, st, lo, hi);
-        if (fuse && d == m - 1) {
-            fused_lo = lo;
-            cur[d] = first(d);
-            end[d] = (hi - lo) * inner_extent;
+        loop_range(LA, b, st, lo, hi);
+        const int32_t f = first(dl), stp = step(dl);
+        if (!s.fast) {                                                    // an operand is located per iteration
+            if (fuse) {
+                const int32_t total = (hi - lo) * inner_extent;
+                for (int32_t c = f; c < total; c += stp) {
+                    if (!bind(LA, b, st, lo + c / inner_extent)) continue;
+                    bind(LB, b, st, c % inner_extent);
+                    update<T>(s, p, b, st, scratch);
+                }
+            } else {
+                for (int32_t it = lo + f; it < hi; it += stp)
+                    if (bind(LB, b, st, it)) update<T>(s, p, b, st, scratch);
+            }
+            return;
+        }
+        // No operand is located here: every reference is affine in the two coordinates and positions
+        // (Stmt::sA, sB, pA, pB), so the loop needs no bindings and no index-by-index addresses.
+        st.idx[LB.index] = 0;
+        if (fuse) st.idx[LA.index] = 0;
+        const Ref *refs[3] = {&s.out, &s.lhs, &s.rhs};
+        const T *ptr[3];
+        int64_t base[3];
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const Ref &ref = *refs[r];
+            if (ref.kind == kRefSparse) {
+                const SparsePtrs &sp = b.sp[ref.slot];
+                ptr[r] = static_cast<const T *>(sp.vals);
+                base[r] = (s.pA[r] | s.pB[r]) ? 0 : st.node[ref.slot][sp.order - 1];
+            } else {
+                ptr[r] = ref.kind == kRefPrivate ? scratch + p.ws[ref.slot].offset : static_cast<const T *>(b.global[ref.slot]);
+                base[r] = address<T>(ref, st);
+            }
+        }
+        T *dst = const_cast<T *>(ptr[0]);
+        const int32_t *crdA = LA.driver >= 0 ? b.sp[LA.driver].crd[LA.level] : nullptr;
+        auto one = [&](int32_t itA, int32_t cA, int32_t itB, int32_t cB) {
+            int64_t at[3];
+#pragma unroll
+            for (int r = 0; r < 3; ++r)
+                at[r] = base[r] + (int64_t)cA * s.sA[r] + (int64_t)cB * s.sB[r] + (int64_t)itA * s.pA[r] + (int64_t)itB * s.pB[r];
+            atomicAdd(dst + at[0], ptr[1][at[1]] * ptr[2][at[2]]);
+        };
+        if (fuse) {
+            const int32_t total = (hi - lo) * inner_extent;
+            int32_t qa = f / inner_extent, qb = f % inner_extent;          // place in the outer range, inner coordinate
+            const int32_t da = stp / inner_extent, db = stp % inner_extent;
+            for (int32_t c = f; c < total; c += stp) {
+                const int32_t itA = lo + qa;
+                one(itA, crdA ? crdA[itA] : itA, 0, qb);
+                qa += da;
+                qb += db;
+                if (qb >= inner_extent) { qb -= inner_extent; ++qa; }
+            }
         } else {
-            cur[d] = lo + first(d);
-            end[d] = hi;
+            for (int32_t it = lo + f; it < hi; it += stp) one(0, 0, it, crdA ? crdA[it] : it);
         }
     };
-    int d = 0;
-    open(0);
-    while (d >= 0) {
-        if (cur[d] >= end[d]) {
-            --d;
-            if (d >= 0) cur[d] += step(d);
-            continue;
-        }
-        bool here;
-        if (fuse && d == m - 1) {
-            here = bind(p.loops[s.priv[d]], b, st, fused_lo + cur[d] / inner_extent);
-            bind(p.loops[s.priv[n - 1]], b, st, cur[d] % inner_extent);
-        } else {
-            here = bind(p.loops[s.priv[d]], b, st, cur[d]);
-        }
-        if (!here) {                                                  // an operand of this assignment is absent
-            cur[d] += step(d);
-            continue;
-        }
-        if (d == m - 1) {
-            update<T>(s, p, b, st, scratch);
-            cur[d] += step(d);
-        } else {
-            ++d;
-            open(d);
+    if (m == 1) {
+        innermost();
+    } else {
+        int d = 0;
+        open(0);
+        while (d >= 0) {
+            if (cur[d] >= end[d]) {
+                --d;
+                if (d >= 0) cur[d] += step(d);
+                continue;
+            }
+            if (!bind(p.loops[s.priv[d]], b, st, cur[d])) {               // an operand of this assignment is absent
+                cur[d] += step(d);
+                continue;
+            }
+            if (d == m - 2) {
+                innermost();
+                cur[d] += step(d);
+            } else {
+                ++d;
+                open(d);
+            }
         }
     }
     // what the private loops bound is dead now; the operands stand where the uniform loops left them

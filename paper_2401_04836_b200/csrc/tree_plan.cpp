@@ -274,6 +274,26 @@ struct Compiler {
         if (s.out.kind == kRefPrivate) s.out.slot = (int8_t)e.ws_id.at(s.out.slot);
         if (s.lhs.kind == kRefPrivate) s.lhs.slot = (int8_t)e.ws_id.at(s.lhs.slot);
         if (s.rhs.kind == kRefPrivate) s.rhs.slot = (int8_t)e.ws_id.at(s.rhs.slot);
+        if (s.n_priv >= 1) {
+            const Loop &LB = e.p.loops[s.priv[s.n_priv - 1]];
+            const Loop *LA = s.fuse_tail ? &e.p.loops[s.priv[s.n_priv - 2]] : nullptr;
+            s.fast = LB.n_follow == 0 && (!LA || LA->n_follow == 0);
+            const TensorRef *names[3] = {&k.out, &k.lhs, &k.rhs};
+            const Ref *refs[3] = {&s.out, &s.lhs, &s.rhs};
+            for (int r = 0; r < 3; ++r) {
+                const Ref &ref = *refs[r];
+                if (ref.kind == kRefSparse) {
+                    const int leaf = (int)tensors.at(names[r]->name).levels.size() - 1;
+                    s.pB[r] = LB.driver == ref.slot && LB.level == leaf;
+                    s.pA[r] = LA && LA->driver == ref.slot && LA->level == leaf;
+                } else {
+                    for (int x = 0; x < ref.n; ++x) {
+                        if (ref.idx[x] == LB.index) s.sB[r] = ref.stride[x];
+                        if (LA && ref.idx[x] == LA->index) s.sA[r] = ref.stride[x];
+                    }
+                }
+            }
+        }
         const Contraction &rk = tree.reduced[c];
         e.stmt_text.push_back(show(rk.out) + " += " + show(rk.lhs) + " * " + show(rk.rhs));
         int at;
