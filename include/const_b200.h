@@ -30,7 +30,7 @@ extern "C" {
 typedef enum {
     CONST_OK = 0,
     CONST_ERR_INVALID_ARG = 1,      /* null pointer, bad order, malformed expression ...               */
-    CONST_ERR_UNSUPPORTED = 2,      /* legal schedule that matches no kernel family, nnz >= 2^31 ...   */
+    CONST_ERR_UNSUPPORTED = 2,      /* beyond a capacity: schedule too large for any executor, nnz >= 2^31 ... */
     CONST_ERR_ILLEGAL_SCHEDULE = 3, /* violates a constraint of Sec. 3.2                               */
     CONST_ERR_DUPLICATE_COORD = 4,  /* the same coordinate tuple appears twice in a COO input          */
     CONST_ERR_COORD_RANGE = 5,      /* a coordinate is negative or >= its extent                       */
@@ -200,7 +200,8 @@ const_status_t const_csf_work_lists(const const_csf_t *csf, const int32_t **slic
  *           example R_ijk = A_ipq B_jpr C_kqr D_jkr with X and Y as 2-D workspaces inside the fused r, j
  *           loops (Fig. 5), order-4 MTTKRP, TTMc at other ranks, the network with U stored (i,j,k) and W
  *           (k,l,m), or a network multiplied by a sparse 0/1 map (Sec. 5.1, Eq. 2).  The outermost loop is
- *           spread over thread blocks; a forall walks the nodes of a CSF operand where skipping the other
+ *           spread over the grid (the two outermost fused loops together when both walk the same CSF
+ *           operand), one iteration per thread block, or per warp when its workspaces are small; a forall walks the nodes of a CSF operand where skipping the other
  *           coordinates cannot change the result, else the dense range of its index, and looks the other CSF
  *           operands up; intermediates are dense workspaces over the indices fusion left them (Sec. 2.2),
  *           cleared at every iteration of the innermost forall shared by producer and consumer.  A producer
