@@ -296,3 +296,26 @@ def test_medium_sizes_reach_every_way_the_iterations_are_dealt_out():
                            w.sparse, w.dense, w.out_shape)
     assert family == "tree"
     assert_close(out, S, A, np.float64)
+
+
+def test_running_example_degenerate_operands():
+    """Each of the four operands empty in turn (the result is exactly zero whichever loop walks or looks up the
+    empty tensor), and every extent equal to one (a single product)."""
+    with open(os.path.join(GOLDEN, "running_example_schedule.json")) as f:
+        g = json.load(f)
+    rng = np.random.default_rng(99)
+    ext = {"i": 5, "j": 6, "k": 4, "p": 5, "q": 3, "r": 4}
+    shape = {"A": "ipq", "B": "jpr", "C": "kqr", "D": "jkr"}
+    full = {t: sparse_input(rng, tuple(ext[x] for x in idx), 40, np.float64) for t, idx in shape.items()}
+    for hollow in shape:
+        dims = tuple(ext[x] for x in shape[hollow])
+        sparse = dict(full)
+        sparse[hollow] = gen.SparseOperand([np.zeros(0, np.int32)] * 3, np.zeros(0, np.float64), dims)
+        out, _ = run_tree(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], ext, cb.F64, sparse, {},
+                          (ext["i"], ext["j"], ext["k"]))
+        assert np.array_equal(out, np.zeros_like(out)), hollow
+    one = {x: 1 for x in ext}
+    vals = {"A": 1.5, "B": -2.0, "C": 0.25, "D": 3.0}
+    sparse = {t: gen.SparseOperand([np.zeros(1, np.int32)] * 3, np.array([v]), (1, 1, 1)) for t, v in vals.items()}
+    out, _ = run_tree(g["expression"], g["tree"], g["mode_orders"], g["loop_orders"], one, cb.F64, sparse, {}, (1, 1, 1))
+    assert out.tolist() == [[[1.5 * -2.0 * 0.25 * 3.0]]]
