@@ -201,7 +201,8 @@ const_status_t const_csf_work_lists(const const_csf_t *csf, const int32_t **slic
  *           loops (Fig. 5), order-4 MTTKRP, TTMc at other ranks, the network with U stored (i,j,k) and W
  *           (k,l,m), or a network multiplied by a sparse 0/1 map (Sec. 5.1, Eq. 2).  The outermost loop is
  *           spread over the grid (the two outermost fused loops together when both walk the same CSF
- *           operand), one iteration per thread block, or per warp when its workspaces are small; a forall walks the nodes of a CSF operand where skipping the other
+ *           operand), one iteration per thread block, or per warp when its workspaces are small; a forall
+ *           walks the nodes of a CSF operand where skipping the other
  *           coordinates cannot change the result, else the dense range of its index, and looks the other CSF
  *           operands up; intermediates are dense workspaces over the indices fusion left them (Sec. 2.2),
  *           cleared at every iteration of the innermost forall shared by producer and consumer.  A producer
